@@ -1,0 +1,223 @@
+"""Pins for the cyclic-code oracle: the paper's lemmas, closed forms, brute force."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import draco_inputs as di
+from oracle import draco_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _exact_sum(G):
+    return G.astype(np.float64).sum(axis=0)
+
+
+def test_W_matches_hand_derived_table_n4_s1():
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "cyc_W_n4_s1.txt")) if not ln.startswith("#")]
+    table = np.array([[0.5 * (float(r[2 * k]) + 1j * float(r[2 * k + 1])) for k in range(4)] for r in rows])
+    np.testing.assert_allclose(orc.cyc_W_by_definition(4, 1), table, atol=1e-15)
+    np.testing.assert_allclose(orc.cyc_W_closed_form(4, 1), table, atol=1e-15)
+
+
+@pytest.mark.parametrize("n,s", [(4, 1), (5, 1), (7, 3), (9, 1), (10, 2), (15, 2), (15, 5), (21, 3)])
+def test_W_definition_equals_closed_form(n, s):
+    Wd, Wc = orc.cyc_W_by_definition(n, s), orc.cyc_W_closed_form(n, s)
+    assert np.abs(Wd - Wc).max() <= 1e-14 * np.abs(Wc).max()
+
+
+def test_W_definition_equals_closed_form_n45_s5():
+    Wd, Wc = orc.cyc_W_by_definition(45, 5, dps=50), orc.cyc_W_closed_form(45, 5)
+    assert np.abs(Wd - Wc).max() <= 1e-14 * np.abs(Wc).max()
+    assert 1.7e5 < np.abs(Wc).max() < 1.9e5               # entries grow geometrically with n and s
+
+
+@pytest.mark.parametrize("n,s", [(4, 1), (9, 2), (15, 2), (45, 5)])
+def test_lemma3_support_and_span(n, s):
+    A, W = orc.cyc_allocation(n, s), orc.cyc_W(n, s)
+    assert A.sum() / n == 2 * s + 1                        # redundancy ratio meets Theorem 1 with equality
+    assert np.abs(W[A == 0]).max() <= 1e-9 * np.abs(W).max()
+    assert np.abs(W[A == 1]).min() > 1e-3
+    rng = np.random.default_rng(n)
+    for trial in range(6):
+        flags = np.zeros(n, dtype=bool)
+        flags[rng.choice(n, size=int(rng.integers(0, 2 * s + 1)), replace=False)] = True
+        for b in (orc.cyc_decode_vector(n, s, flags), orc.cyc_decode_vector_first(n, s, flags)):
+            assert np.all(b[flags] == 0)
+            assert np.abs(W @ b - 1.0).max() <= 1e-7 * np.abs(W).max() * max(1.0, np.abs(b).max())
+    flags = np.zeros(n, dtype=bool)
+    flags[: 2 * s + 1] = True
+    with pytest.raises(ValueError):
+        orc.cyc_decode_vector(n, s, flags)
+
+
+def test_min_norm_vector_lies_in_row_space():
+    n, s = 15, 2
+    flags = np.zeros(n, dtype=bool)
+    flags[[2, 9]] = True
+    b = orc.cyc_decode_vector(n, s, flags)
+    U = np.flatnonzero(~flags)
+    A = orc.idft_matrix(n)[: n - 2 * s][:, U]
+    null = np.linalg.svd(A)[2][n - 2 * s:].conj().T      # basis of the null space of A
+    assert np.abs(null.conj().T @ b[U]).max() < 1e-12      # min-norm <=> orthogonal to the null space
+    assert np.linalg.norm(b) <= np.linalg.norm(orc.cyc_decode_vector_first(n, s, flags)) + 1e-12
+
+
+def test_literal_decode_vector_is_lagrange_closed_form():
+    """b_k = sqrt(n) / prod_{l in U-bar, l != k} (w^k - w^l) solves [C_L]_{., U-bar} b = e_last."""
+    n, s = 15, 2
+    flags = np.zeros(n, dtype=bool)
+    flags[[0, 7]] = True
+    Ubar = np.flatnonzero(~flags)[: n - 2 * s]
+    w = np.exp(2j * np.pi / n)
+    expect = np.zeros(n, dtype=complex)
+    for k in Ubar:
+        expect[k] = np.sqrt(n) / np.prod([w ** k - w ** l for l in Ubar if l != k])
+    np.testing.assert_allclose(orc.cyc_decode_vector_first(n, s, flags), expect, rtol=1e-9, atol=1e-12)
+
+
+@pytest.mark.parametrize("n,s", [(4, 1), (15, 2), (45, 5)])
+def test_lemma7_orthogonality_and_clean_syndromes(n, s):
+    C = orc.idft_matrix(n)
+    np.testing.assert_allclose(C @ C.conj().T, np.eye(n), atol=1e-13)       # unitary
+    np.testing.assert_allclose(C, C.T, atol=0)                              # symmetric
+    C_L, C_R = C[: n - 2 * s], C[n - 2 * s:]
+    assert np.abs(C_L @ C_R.conj().T).max() < 1e-13
+    d = 64
+    G = di.gradient_rows(1, n, d)
+    Z = orc.cyc_encode(G, n, s, dtype=np.complex128)
+    synd = Z.T @ C_R.conj().T                                               # R C_R^dagger, per coordinate
+    assert np.abs(synd).max() <= 1e-10 * np.abs(Z).max()
+    f = di.projection_vector(2, d)
+    loc = orc.cyc_locate(Z, f, n, s)
+    assert not loc["flags"].any() and loc["rank"] == 0
+
+
+@pytest.mark.parametrize("n,s", [(4, 1), (15, 2), (45, 5), (45, 3)])
+def test_locator_returns_f_times_N_value_for_value(n, s):
+    """Proof of Lemma 4: t = C h = gamma = (f N)^T, for 0..s adversaries."""
+    d = 200
+    G = di.gradient_rows(21, n, d)
+    Z = orc.cyc_encode(G, n, s, dtype=np.complex128)
+    f = di.projection_vector(22, d)
+    rng = np.random.default_rng(5)
+    for a in range(s + 1):
+        adv = np.sort(rng.choice(n, size=a, replace=False))
+        N = np.zeros_like(Z)
+        N[adv] = (rng.normal(size=(a, d)) + 1j * rng.normal(size=(a, d))) * 50.0 * np.abs(Z).max()
+        loc = orc.cyc_locate(Z + N, f, n, s)
+        gamma = N @ f.astype(np.float64)
+        assert loc["rank"] == a
+        assert set(np.flatnonzero(loc["flags"])) == set(adv.tolist())
+        if a:
+            assert np.abs(loc["t"] - gamma).max() <= 1e-6 * np.abs(gamma).max()
+
+
+@pytest.mark.parametrize("n,s", [(3, 1), (4, 1), (5, 1), (5, 2), (6, 2), (7, 3), (9, 2), (10, 1), (15, 2)])
+def test_every_placement_of_up_to_s_adversaries_is_corrected(n, s):
+    """Definition 2 / Theorem 5 by brute force on tiny n (complex128 transport)."""
+    d = 16
+    G = di.gradient_rows(31, n, d)
+    Z = orc.cyc_encode(G, n, s, dtype=np.complex128)
+    f = di.projection_vector(32, d)
+    exact = _exact_sum(G)
+    attacks = [(di.ADV_REVGRAD, 100.0), (di.ADV_CONST, -100.0), (di.ADV_GAUSS, 1e3)]
+    for a in range(s + 1):
+        for placement in itertools.combinations(range(n), a):
+            for model, param in attacks:
+                R = Z.copy().astype(np.complex64)          # the corruptor works on complex64 rows
+                di.apply_adversaries(R, placement, [model] * a, [param] * a, seed=3)
+                R = R.astype(np.complex128)
+                honest = np.setdiff1d(np.arange(n), placement)
+                R[honest] = Z[honest]                      # honest rows keep full precision
+                out = orc.cyc_decode_full(R, f, n, s)
+                assert set(np.flatnonzero(out["flags"])) == set(placement), (placement, model)
+                assert np.abs(out["u"] - exact).max() <= 1e-8 * np.abs(exact).max()
+    # a single corrupted coordinate on one node
+    R = Z.copy()
+    R[n - 1, 5] += 3.0
+    out = orc.cyc_decode_full(R, f, n, s)
+    assert list(np.flatnonzero(out["flags"])) == [n - 1]
+    assert np.abs(out["u"] - exact).max() <= 1e-8 * np.abs(exact).max()
+
+
+def test_failure_beyond_s():
+    """Theorem 1 / its corollary: s + 1 adversaries defeat a redundancy-(2 s + 1) code."""
+    n, s, d = 15, 2, 32
+    G = di.gradient_rows(41, n, d)
+    Z = orc.cyc_encode(G, n, s, dtype=np.complex128)
+    f = di.projection_vector(42, d)
+    exact = _exact_sum(G)
+    failures = 0
+    placements = list(itertools.combinations(range(n), s + 1))[::7]
+    for placement in placements:
+        R = Z.copy()
+        R[list(placement)] *= -100.0
+        out = orc.cyc_decode_full(R, f, n, s)
+        ok = (set(np.flatnonzero(out["flags"])) == set(placement) and out["u"] is not None
+              and np.abs(out["u"] - exact).max() <= 1e-6 * np.abs(exact).max())
+        failures += not ok
+    assert failures == len(placements)
+
+
+def test_n4_any_two_coded_vectors_recover_the_sum():
+    """Figure 1: 4 gradients, replication 3, any 2 coded vectors give the sum; a
+    majority vote over the 6 pair-decodes survives one adversary."""
+    n, s, d = 4, 1, 8
+    G = di.gradient_rows(51, n, d)
+    Z = orc.cyc_encode(G, n, s, dtype=np.complex128)
+    exact = _exact_sum(G)
+    pairs = list(itertools.combinations(range(n), 2))
+    assert len(pairs) == 6
+    for pair in pairs:
+        flags = np.ones(n, dtype=bool)
+        flags[list(pair)] = False
+        np.testing.assert_allclose(orc.cyc_decode(Z, n, s, flags), exact, atol=1e-12)
+    R = Z.copy()
+    R[2] = -100.0 * R[2]
+    decodes = []
+    for pair in pairs:
+        flags = np.ones(n, dtype=bool)
+        flags[list(pair)] = False
+        decodes.append(np.round(orc.cyc_decode(R, n, s, flags), 9))
+    agree = [sum(np.array_equal(x, y) for y in decodes) for x in decodes]
+    assert sorted(agree) == [1, 1, 1, 3, 3, 3]              # 3 clean pairs agree, 3 dirty pairs differ
+    winner = decodes[int(np.argmax(agree))]
+    np.testing.assert_allclose(winner, exact, atol=1e-8)
+    f = di.projection_vector(52, d)
+    np.testing.assert_allclose(orc.cyc_decode_full(R, f, n, s)["u"], exact, atol=1e-10)
+
+
+def test_no_adversary_decode_vector_is_conjugate_idft_row():
+    for n, s in [(4, 1), (15, 2), (45, 5)]:
+        b = orc.cyc_decode_vector(n, s, np.zeros(n, dtype=bool))
+        np.testing.assert_allclose(b, orc.idft_matrix(n)[n - 2 * s - 1].conj(), atol=1e-12)
+        G = di.gradient_rows(61, n, 50)
+        Z = orc.cyc_encode(G, n, s, dtype=np.complex128)
+        uhat = orc.cyc_recover(Z, b)
+        scale = np.abs(orc.cyc_W(n, s)).max()
+        assert np.abs(uhat.real - _exact_sum(G)).max() <= 1e-12 * scale * 10
+        assert np.abs(uhat.imag).max() <= 1e-12 * scale * 10          # Im(u-hat) is rounding residue
+
+
+def test_full_redundancy_degenerates_to_repetition():
+    n, s = 15, 7                                           # r = n: C_L has one row
+    W = orc.cyc_W(n, s)
+    np.testing.assert_allclose(W, np.full((n, n), 1 / np.sqrt(n)), atol=1e-14)
+
+
+def test_complex64_transport_floor():
+    """With complex64 worker vectors the recovered sum is only as good as the
+    code's cancellation allows: tight at (15,2), about 1e-3 at (45,5)."""
+    for (n, s, lo, hi) in [(15, 2, 0.0, 5e-6), (45, 5, 1e-4, 1e-2)]:
+        d = 4000
+        G = di.gradient_rows(71, n, d)
+        R = orc.cyc_encode(G, n, s)
+        adv = di.choose_adversaries(72, n, s)
+        di.apply_adversaries(R, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=0)
+        out = orc.cyc_decode_full(R, di.projection_vector(73, d), n, s)
+        assert list(np.flatnonzero(out["flags"])) == adv.tolist()
+        err = np.abs(out["u"] - _exact_sum(G)).max() / np.abs(_exact_sum(G)).max()
+        assert lo <= err <= hi, err
