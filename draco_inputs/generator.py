@@ -63,15 +63,22 @@ def _sum16(h):
     return s
 
 
+_BLOCK = 1 << 16  # elements per pass: keeps the temporaries cache-resident
+
+
 def approx_normal_at(seed: int, row: int, idx) -> np.ndarray:
     """Standard-normal-like float32 values of row ``row`` at coordinates ``idx``."""
     idx = np.asarray(idx, dtype=np.uint64)
     key = row_key(seed, row)
-    with np.errstate(over="ignore"):
-        c0 = idx * np.uint64(2)
-        s = _sum16(splitmix64_at(key, c0)) + _sum16(splitmix64_at(key, c0 + np.uint64(1)))
-    centred = s.astype(np.int64) - np.int64(IH_CENTER)
-    return centred.astype(np.float32) * INV_SIGMA_F32
+    out = np.empty(idx.shape[0], dtype=np.float32)
+    for b0 in range(0, idx.shape[0], _BLOCK):
+        part = idx[b0:b0 + _BLOCK]
+        with np.errstate(over="ignore"):
+            c0 = part * np.uint64(2)
+            s = _sum16(splitmix64_at(key, c0)) + _sum16(splitmix64_at(key, c0 + np.uint64(1)))
+        centred = s.astype(np.int64) - np.int64(IH_CENTER)
+        out[b0:b0 + _BLOCK] = centred.astype(np.float32) * INV_SIGMA_F32
+    return out
 
 
 def approx_normal_rows(seed: int, rows, i0: int, i1: int, mean: float = 0.0, std: float = 1.0,

@@ -1,0 +1,180 @@
+/*
+ * draco.h - C ABI of the B200 (sm_100a) implementation of the parameter-server
+ * hot path of Draco (arXiv 1803.09877): redundant-gradient encoding, adversary
+ * location and exact decoding for the repetition code and the cyclic code.
+ *
+ * Notation (the paper's, Section 3):  n = P compute nodes (= B gradients),
+ * s = number of adversarial nodes tolerated, r = 2 s + 1 the redundancy ratio,
+ * d = gradient dimension, G = [g_1 .. g_P], z_j = E_j(Y_j) what node j sends,
+ * R = Z + N what the parameter server receives, u = D(R).
+ *
+ * Layout.  Every matrix is worker-major and dense: row k of G is gradient g_k
+ * (d contiguous fp32), row j of Z / R is node j's vector: d fp32 for the
+ * repetition code, d interleaved (re, im) fp32 pairs (complex64) for the cyclic
+ * code.  u is d fp32.  Indices are 0-based.  Row stride = d elements.
+ *
+ * Ownership.  The caller owns every buffer it passes (device buffers unless a
+ * parameter says "host"); the library never frees or keeps them.  A plan owns
+ * its code tables and a small device scratch area allocated by
+ * draco_plan_create (kilobytes to a few hundred kilobytes), released by
+ * draco_plan_destroy.  Device pointers must be 16-byte aligned.
+ *
+ * Streams.  `stream` is a cudaStream_t passed as void* (NULL = the default
+ * stream).  Calls enqueue work and return without synchronising unless stated.
+ * Calls on one plan must not overlap on the device (they share its scratch).
+ *
+ * Errors.  Functions return DRACO_OK (0) or a negative DRACO_E* code; nothing
+ * throws or aborts.  Conditions found on the device (too many nodes flagged, no
+ * strict majority somewhere) are reported through draco_get_info.
+ */
+#ifndef DRACO_H_
+#define DRACO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct draco_plan draco_plan;
+
+/* code type */
+enum { DRACO_REP = 0, DRACO_CYC = 1 };
+/* adversary models of the corruptor (Section 4, "Adversarial Attack Models", plus Gaussian noise) */
+enum { DRACO_ADV_REVGRAD = 0, DRACO_ADV_CONST = 1, DRACO_ADV_GAUSS = 2 };
+/* return codes */
+enum {
+    DRACO_OK = 0,
+    DRACO_EINVAL = -1,   /* bad argument: n < 1, s < 0, 2 s + 1 > n (Corollary of Theorem 1), null or misaligned pointer */
+    DRACO_ECUDA = -2,    /* a CUDA runtime call failed (see draco_last_cuda_error) */
+    DRACO_ETOOMANY = -3, /* more than 2 s nodes flagged: no decode vector exists (u is written as zeros) */
+    DRACO_ENOMEM = -4,
+    DRACO_ENOMAJ = 1     /* warning: some (group, coordinate) had no strict majority; u holds Algorithm 2's candidate */
+};
+
+#define DRACO_MAX_N 128  /* largest supported number of nodes */
+
+/* Device-side results of the most recent locate / decode on a plan. */
+typedef struct draco_info {
+    int32_t status;        /* DRACO_OK, DRACO_ETOOMANY or DRACO_ENOMAJ */
+    int32_t n_flagged;     /* |V|: nodes flagged by the last locate (or given to the last cyclic decode) */
+    int32_t locator_rank;  /* cyclic: numerical rank of the s x s syndrome system = adversaries seen */
+    int32_t n_active;      /* cyclic decode: number of rows with b_j != 0 */
+    uint64_t no_majority;  /* repetition: (group, coordinate) pairs without a strict majority */
+    double scale;          /* cyclic: median_j |e_j| of the projection, the unit of the threshold */
+    double max_syndrome;   /* cyclic: max_m |h_m| over the 2 s syndromes */
+} draco_info;
+
+/*
+ * Build the tables for one (n, s, d, code) and allocate the plan's scratch on
+ * the current CUDA device.  Repetition code (Section 3, "Fractional Repetition
+ * Code"): groups of consecutive nodes; n / r groups of r when r divides n,
+ * otherwise floor(n / r) groups whose sizes differ by at most one (all >= r).
+ * Cyclic code (Section 3, "Cyclic Code"): the matrix W = [Q 1_P] C_L in closed
+ * form, the IDFT twiddles, and the locator / decode-vector work space.
+ * Requires 1 <= n <= DRACO_MAX_N, s >= 0, 2 s + 1 <= n, d >= 1.
+ */
+int draco_plan_create(int n, int s, int64_t d, int code, draco_plan** out);
+int draco_plan_destroy(draco_plan* plan);
+
+/* Rank cutoff theta of the cyclic locator (default 1e-6): singular values of the s x s syndrome
+ * system below theta * median_j |e_j| count as zero.  The rank found is the number of adversaries
+ * seen, and V is the set of that many nodes with the largest |t_j| (exactly that many t_j are
+ * non-zero in exact arithmetic). */
+int draco_plan_set_theta(draco_plan* plan, double theta);
+
+/* Number of groups of a repetition plan (0 for a cyclic plan); group g covers
+ * nodes first[g] .. first[g] + size[g] - 1 (host arrays of draco_num_groups entries, may be NULL). */
+int draco_num_groups(const draco_plan* plan);
+int draco_groups(const draco_plan* plan, int* first /*host*/, int* size /*host*/);
+
+/* Cyclic plans: copy W (n x n complex, row-major, (re, im) doubles; z_j = sum_k W[k][j] g_k) to host memory. */
+int draco_cyc_W(const draco_plan* plan, double* W_host /*host [n][n][2]*/);
+
+/*
+ * Encoding: Z[j] = E_j(Y_j) for all n nodes in one pass over G.
+ *   repetition: z_j = Y_j 1_P = sum of the gradients of j's group, ascending, fp32
+ *               (members of a group produce identical bits);
+ *   cyclic:     z_j = G W_{.,j} = sum_{t=0..2s} W[j-t][j] g_{(j-t) mod n}, complex64.
+ * G: device [n][d] fp32.  Z: device [n][d] fp32 (repetition) or complex64 (cyclic).
+ */
+int draco_encode(const draco_plan* plan, const float* G, void* Z, void* stream);
+
+/*
+ * Locating the adversaries: flags[j] = 1 iff node j is in V, else 0.
+ *   repetition: j is flagged when its vector differs in any bit, at any coordinate,
+ *               from the majority of its group (derived from D^Rep; f is ignored);
+ *   cyclic:     V = phi(R): e = f R (fp64 accumulation), the 2 s syndromes e C_R^dagger,
+ *               the s x s Toeplitz system for beta (pseudo-inverse solution from an SVD),
+ *               the recurrence h_l = sum_u beta_u h_{l+u-s}, t = IDFT(h), V = supp(t)
+ *               read as the rank-many largest |t_j|.
+ * R: device [n][d].  f: device [d] fp32, the caller's draw of N(1_d, I_d) (cyclic only).
+ * flags: device [n] bytes.
+ */
+int draco_locate(draco_plan* plan, const void* R, const float* f, uint8_t* flags, void* stream);
+
+/*
+ * Decoding: u = D(R).
+ *   repetition: u = sum over groups of Maj(group) (Algorithm 2 on 32-bit patterns), groups
+ *               ascending, fp32; flags may be NULL and is ignored;
+ *   cyclic:     Algorithm 1, steps 2-4: U = nodes with flags[j] = 0, b = the minimum-norm
+ *               solution of W_{.,U} b = 1_P, u = Re(R_{.,U} b), fp64 accumulation, fp32 result.
+ * flags: device [n] bytes (cyclic: required).  u: device [d] fp32.
+ */
+int draco_decode(draco_plan* plan, const void* R, const uint8_t* flags, float* u, void* stream);
+
+/* locate + decode in one call (repetition: one pass over R; cyclic: locate, then decode). */
+int draco_locate_decode(draco_plan* plan, const void* R, const float* f, uint8_t* flags, float* u, void* stream);
+
+/* Repetition code with the selections exposed: maj (device [groups][d] fp32, may be NULL) receives
+ * the value selected for every group and coordinate; u and flags may be NULL. */
+int draco_rep_vote(draco_plan* plan, const void* R, float* u, float* maj, uint8_t* flags, void* stream);
+
+/* The two halves of the cyclic locator, for callers that shard d across devices and add the
+ * projections: e (device [n] complex as (re, im) doubles) = f R over this plan's d coordinates. */
+int draco_cyc_project(draco_plan* plan, const void* R, const float* f, double* e, void* stream);
+int draco_cyc_locate_from_projection(draco_plan* plan, const double* e, uint8_t* flags, void* stream);
+
+/* The decode vector b of the last cyclic decode (host [n][2] doubles); synchronises the stream. */
+int draco_cyc_decode_vector(draco_plan* plan, double* b_host /*host*/, void* stream);
+
+/* Copies the device-side results of the last calls to host memory; synchronises the stream. */
+int draco_get_info(draco_plan* plan, draco_info* info /*host*/, void* stream);
+
+/*
+ * Whole path with host buffers (pageable or pinned): copies G and f to the device in
+ * column chunks, encodes, applies the given adversaries, locates, decodes, and copies
+ * u and flags back.  Synchronous.  Z (device [n][d], caller-owned) keeps the received matrix.
+ */
+int draco_pipeline_host(draco_plan* plan, const float* G_host, const float* f_host,
+                        const int* adv_idx /*host*/, const int* adv_model /*host*/, const float* adv_param /*host*/,
+                        int n_adv, uint64_t adv_seed, void* Z, float* u_host, uint8_t* flags_host,
+                        draco_info* info /*host, may be NULL*/);
+
+/*
+ * Seeded synthetic inputs (counter-based; identical bits to the published definition:
+ * row key = SplitMix64 output number row+1 from state seed; element i of a row sums the eight
+ * 16-bit fields of outputs 2 i + 1 and 2 i + 2 from state key, S; value =
+ * fl32(fl32(fl32(S - 262140) * c) * std) + mean with c = fl32(1 / sqrt(8 (2^32 - 1) / 12))).
+ * out: device [rows][len] fp32, rows numbered row0 .. row0 + rows - 1.
+ */
+int draco_generate(float* out, int rows, int64_t len, int row0, float mean, float std, uint64_t seed, void* stream);
+
+/*
+ * The adversary: R = Z + N in place, N non-zero on rows adv_idx[0 .. n_adv-1] (host arrays).
+ *   DRACO_ADV_REVGRAD: row <- -c * row          (param = c)
+ *   DRACO_ADV_CONST:   row <- kappa             (param = kappa; imaginary parts 0)
+ *   DRACO_ADV_GAUSS:   row <- row + sigma * x   (param = sigma; x from the generator above with
+ *                      seed `seed`, row = node index, over the row's fp32 values)
+ */
+int draco_corrupt(const draco_plan* plan, void* R, const int* adv_idx, const int* adv_model,
+                  const float* adv_param, int n_adv, uint64_t seed, void* stream);
+
+const char* draco_strerror(int code);
+/* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
+const char* draco_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DRACO_H_ */

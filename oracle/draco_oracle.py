@@ -20,8 +20,9 @@ Algorithm 2 against sort-and-count; the adversary-free decode reducing to a
 plain sum.
 
 Parity unpinned (readings, not paper facts; they do not change the exact
-result): the detection threshold ``theta``; the grouping used when 2 s + 1 does
-not divide n; the minimum-norm choice among the valid decode vectors b.
+result): the rank cutoff ``theta`` of the locator and its "rank largest |t_j|"
+reading of t_j != 0; the grouping used when 2 s + 1 does not divide n; the
+minimum-norm choice among the valid decode vectors b.
 """
 from __future__ import annotations
 
@@ -243,7 +244,7 @@ def cyc_project(R: np.ndarray, f: np.ndarray) -> np.ndarray:
     return np.asarray(R, dtype=np.complex128) @ np.asarray(f, dtype=np.float64)
 
 
-def cyc_locate_from_projection(e: np.ndarray, n: int, s: int, theta: float = 1e-4) -> dict:
+def cyc_locate_from_projection(e: np.ndarray, n: int, s: int, theta: float = 1e-6) -> dict:
     """The locator phi after the projection: syndromes, Toeplitz solve,
     recurrence, IDFT, support.
 
@@ -252,27 +253,28 @@ def cyc_locate_from_projection(e: np.ndarray, n: int, s: int, theta: float = 1e-
       * row i of the s x s system is [h_{n-s-1-i} .. h_{n-2-i}] with right-hand
         side h_{n-1-i}: the recurrence h_l = sum_u beta_u h_{l+u-s} written for
         l = n-1-i;
-      * fewer than s adversaries make the system singular: singular values below
-        theta * scale are dropped (pseudo-inverse); Lemma 8 lets any solution
-        of the equations drive the recurrence;
-      * "t_j != 0" is read as |t_j| > theta * scale with scale = median_j |e_j|
-        (at least n - s rows are honest); if every syndrome is within
-        theta * scale of zero, V is empty.
+      * fewer than s adversaries make the system singular (its rank is the
+        number of non-zero entries of gamma = (f N)^T): singular values below
+        theta * scale, scale = median_j |e_j|, count as zero and beta is the
+        pseudo-inverse solution; Lemma 8 lets any solution of the equations
+        drive the recurrence;
+      * "t_j != 0" cannot be tested in floating point.  Exactly ``rank`` entries
+        of t are non-zero in exact arithmetic, so V = the ``rank`` nodes with the
+        largest |t_j| (V is empty when the rank is 0).
     """
     e = np.asarray(e, dtype=np.complex128)
     C = idft_matrix(n)
     scale = float(np.median(np.abs(e)))
     tol = theta * scale
     out = {"e": e, "scale": scale, "t": np.zeros(n, dtype=np.complex128),
-           "flags": np.zeros(n, dtype=bool), "rank": 0, "h": np.zeros(n, dtype=np.complex128)}
+           "flags": np.zeros(n, dtype=bool), "rank": 0, "h": np.zeros(n, dtype=np.complex128),
+           "margin": np.inf}
     if s == 0:
         return out
     C_R = C[n - 2 * s:]
     h = np.zeros(n, dtype=np.complex128)
     h[n - 2 * s:] = e @ C_R.conj().T
     out["h"] = h
-    if np.max(np.abs(h[n - 2 * s:])) <= tol:
-        return out
     M = np.empty((s, s), dtype=np.complex128)
     rhs = np.empty(s, dtype=np.complex128)
     for i in range(s):
@@ -282,6 +284,9 @@ def cyc_locate_from_projection(e: np.ndarray, n: int, s: int, theta: float = 1e-
     Us, sv, Vh = np.linalg.svd(M)
     keep = sv > tol
     rank = int(np.count_nonzero(keep))
+    out["sv"] = sv
+    if rank == 0:
+        return out
     inv = np.zeros_like(sv)
     inv[keep] = 1.0 / sv[keep]
     beta = Vh.conj().T @ (inv * (Us.conj().T @ rhs))
@@ -291,11 +296,15 @@ def cyc_locate_from_projection(e: np.ndarray, n: int, s: int, theta: float = 1e-
             acc += beta[u] * h[(ell + u - s) % n]
         h[ell] = acc
     t = C @ h
-    out.update(h=h, t=t, flags=np.abs(t) > tol, rank=rank, beta=beta)
+    order = np.argsort(-np.abs(t), kind="stable")
+    flags = np.zeros(n, dtype=bool)
+    flags[order[:rank]] = True
+    margin = np.abs(t[order[rank - 1]]) / max(np.abs(t[order[rank]]), 1e-300) if rank < n else np.inf
+    out.update(h=h, t=t, flags=flags, rank=rank, beta=beta, margin=float(margin))
     return out
 
 
-def cyc_locate(R: np.ndarray, f: np.ndarray, n: int, s: int, theta: float = 1e-4) -> dict:
+def cyc_locate(R: np.ndarray, f: np.ndarray, n: int, s: int, theta: float = 1e-6) -> dict:
     """V = phi(R) with the random vector f passed in (f ~ N(1_d, I_d))."""
     return cyc_locate_from_projection(cyc_project(R, f), n, s, theta)
 
@@ -350,7 +359,7 @@ def cyc_decode(R: np.ndarray, n: int, s: int, flags, literal_b: bool = False) ->
     return cyc_recover(R, b).real
 
 
-def cyc_decode_full(R: np.ndarray, f: np.ndarray, n: int, s: int, theta: float = 1e-4) -> dict:
+def cyc_decode_full(R: np.ndarray, f: np.ndarray, n: int, s: int, theta: float = 1e-6) -> dict:
     """Algorithm 1 in full: locate, then decode."""
     loc = cyc_locate(R, f, n, s, theta)
     loc["u"] = cyc_decode(R, n, s, loc["flags"]) if loc["flags"].sum() <= 2 * s else None

@@ -1,0 +1,547 @@
+// Cyclic-code adversary locator phi(R) (Section 3, "Cyclic Code"; correctness: Lemmas 4, 6-8).
+//
+//   cyc_project_kernel   e_j = sum_i f_i R[j][i]: the one O(d P) step, a single pass over R.
+//   cyc_solve_kernel     [h_{n-2s} .. h_{n-1}] = e C_R^dagger, the s x s Toeplitz system for
+//                        beta (pseudo-inverse by a Jacobi SVD: its rank = the number of
+//                        adversaries seen), the recurrence h_l = sum_u beta_u h_{l+u-s}, t = C h,
+//                        V = the `rank` nodes with the largest |t_j|.
+//   cyc_decode_vector_kernel   b with support in U = [n] \ V and [C_L]_{.,U} b_U = (0,..,0,1)^T
+//                        (equivalent to W_{.,U} b = 1_P, proof of Lemma 3), minimum 2-norm.
+//
+// The small solves run in fp64 in a single thread block; only the projection touches HBM:
+// 8 n len + 4 len bytes read.
+#include "draco_internal.cuh"
+
+namespace draco {
+
+namespace {
+
+constexpr int kThreads = kProjectWarps * 32;
+constexpr int kSolveThreads = 128;
+
+__device__ __forceinline__ double2 cmul(double2 a, double2 b) {
+    return make_double2(a.x * b.x - a.y * b.y, a.x * b.y + a.y * b.x);
+}
+__device__ __forceinline__ double2 cmulc(double2 a, double2 b) {   // a * conj(b)
+    return make_double2(a.x * b.x + a.y * b.y, a.y * b.x - a.x * b.y);
+}
+__device__ __forceinline__ double2 cdiv(double2 a, double2 b) {
+    const double den = b.x * b.x + b.y * b.y;
+    const double2 q = cmulc(a, b);
+    return make_double2(q.x / den, q.y / den);
+}
+__device__ __forceinline__ double cabs2(double2 a) { return a.x * a.x + a.y * a.y; }
+
+// ------------------------------------------------------------------ projection
+// Block = 8 warps over one tile of coordinates; warp w owns rows w, w+8, ...; f for the tile
+// sits in shared memory.  Products and short runs (16 terms) in fp32, running sums in fp64.
+template <int RPW, bool VEC2>
+__global__ void __launch_bounds__(kThreads)
+cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
+                   double2* __restrict__ partial, int accumulate) {
+    __shared__ __align__(16) float fs[kProjectTile];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    double accr[RPW], acci[RPW];
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) { accr[r] = 0.0; acci[r] = 0.0; }
+
+    const int64_t ntiles = (len + kProjectTile - 1) / kProjectTile;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int64_t c0 = tile * kProjectTile;
+        const int cnt = (int)((len - c0) < kProjectTile ? (len - c0) : kProjectTile);
+        for (int i = threadIdx.x; i < kProjectTile; i += kThreads) fs[i] = (i < cnt) ? __ldcs(f + c0 + i) : 0.0f;
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+            const int j = warp + r * kProjectWarps;
+            if (j < n) {
+                const float2* row = R + (int64_t)j * ld + c0;
+                if (VEC2 && cnt == kProjectTile) {
+                    const float4* row4 = reinterpret_cast<const float4*>(row);
+#pragma unroll 1
+                    for (int step0 = 0; step0 < kProjectTile / 64; step0 += 8) {
+                        float4 v[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) v[q] = __ldcs(row4 + (step0 + q) * 32 + lane);
+                        float pr = 0.f, pi = 0.f;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const float2 ff = *reinterpret_cast<const float2*>(&fs[((step0 + q) * 32 + lane) * 2]);
+                            pr = fmaf(ff.x, v[q].x, pr); pi = fmaf(ff.x, v[q].y, pi);
+                            pr = fmaf(ff.y, v[q].z, pr); pi = fmaf(ff.y, v[q].w, pi);
+                        }
+                        accr[r] += (double)pr;
+                        acci[r] += (double)pi;
+                    }
+                } else {
+                    for (int i = lane; i < cnt; i += 32) {
+                        const float2 v = __ldcs(row + i);
+                        const float ff = fs[i];
+                        accr[r] += (double)(ff * v.x);
+                        acci[r] += (double)(ff * v.y);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) {
+        double a = accr[r], b = acci[r];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, off);
+            b += __shfl_xor_sync(0xffffffffu, b, off);
+        }
+        const int j = warp + r * kProjectWarps;
+        if (lane == 0 && j < n) {
+            double2* dst = partial + (int64_t)blockIdx.x * n + j;
+            if (accumulate) { a += dst->x; b += dst->y; }
+            *dst = make_double2(a, b);
+        }
+    }
+}
+
+// e_j = sum over blocks, fixed order.
+__global__ void cyc_project_finish_kernel(const double2* __restrict__ partial, int grid, int n, double2* e) {
+    const int j = threadIdx.x;
+    if (j < n) {
+        double a = 0.0, b = 0.0;
+        for (int blk = 0; blk < grid; ++blk) {
+            const double2 p = partial[(int64_t)blk * n + j];
+            a += p.x;
+            b += p.y;
+        }
+        e[j] = make_double2(a, b);
+    }
+}
+
+// ------------------------------------------------------------------ small dense solve
+// Gauss-Jordan elimination with complete pivoting on the dim x (dim+1) augmented matrix A
+// (row stride dim+1) by one thread block.  Pivots with |pivot| <= tol end the elimination
+// (numerical rank); the free unknowns are set to zero.  x receives the solution.
+__device__ int block_gauss_jordan(double2* A, int dim, double tol, double2* x, int* perm, double* rowbest,
+                                  int* rowbestc, int* sh) {
+    const int tid = threadIdx.x, ldA = dim + 1;
+    for (int i = tid; i < dim; i += blockDim.x) perm[i] = i;
+    __syncthreads();
+    int rank = 0;
+    for (int p = 0; p < dim; ++p) {
+        for (int i = p + tid; i < dim; i += blockDim.x) {
+            double best = -1.0;
+            int bc = p;
+            for (int c = p; c < dim; ++c) {
+                const double m = cabs2(A[i * ldA + c]);
+                if (m > best) { best = m; bc = c; }
+            }
+            rowbest[i] = best;
+            rowbestc[i] = bc;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double best = -1.0;
+            int br = p;
+            for (int i = p; i < dim; ++i)
+                if (rowbest[i] > best) { best = rowbest[i]; br = i; }
+            sh[0] = br;
+            sh[1] = rowbestc[br];
+            sh[2] = (best > tol * tol) ? 1 : 0;
+        }
+        __syncthreads();
+        const int pr = sh[0], pc = sh[1], ok = sh[2];
+        if (!ok) break;
+        if (pr != p)
+            for (int c = tid; c <= dim; c += blockDim.x) {
+                const double2 tmp = A[p * ldA + c];
+                A[p * ldA + c] = A[pr * ldA + c];
+                A[pr * ldA + c] = tmp;
+            }
+        __syncthreads();
+        if (pc != p) {
+            for (int i = tid; i < dim; i += blockDim.x) {
+                const double2 tmp = A[i * ldA + p];
+                A[i * ldA + p] = A[i * ldA + pc];
+                A[i * ldA + pc] = tmp;
+            }
+            if (tid == 0) { const int tmp = perm[p]; perm[p] = perm[pc]; perm[pc] = tmp; }
+        }
+        __syncthreads();
+        const double2 piv = A[p * ldA + p];
+        for (int i = tid; i < dim; i += blockDim.x) {
+            if (i == p) continue;
+            const double2 factor = cdiv(A[i * ldA + p], piv);
+            for (int c = p + 1; c <= dim; ++c) {
+                const double2 q = cmul(factor, A[p * ldA + c]);
+                A[i * ldA + c].x -= q.x;
+                A[i * ldA + c].y -= q.y;
+            }
+            A[i * ldA + p] = make_double2(0.0, 0.0);
+        }
+        __syncthreads();
+        rank = p + 1;
+    }
+    __syncthreads();
+    for (int i = tid; i < dim; i += blockDim.x) x[i] = make_double2(0.0, 0.0);
+    __syncthreads();
+    for (int k = tid; k < rank; k += blockDim.x) x[perm[k]] = cdiv(A[k * ldA + dim], A[k * ldA + k]);
+    __syncthreads();
+    return rank;
+}
+
+// ------------------------------------------------------------------ small SVD solve
+// Pseudo-inverse solution of the s x s complex system A beta = rhs by one-sided (Hestenes)
+// Jacobi: columns of [A; V] are rotated in pairs until the columns of A are orthogonal; then
+// A = U Sigma, sigma_k = |a_k|, and beta = sum_{sigma_k > tol} v_k (a_k^H rhs) / sigma_k^2.
+// Singular values come out to high relative accuracy, so the rank decision (sigma_k > tol)
+// matches a LAPACK SVD except on a knife edge.  A, V: column-major with column stride ld
+// (ld = s rounded up to even; a zero pad column never rotates).  One thread per column pair,
+// pairs of a step disjoint (round-robin schedule).  Returns the rank.
+__device__ int block_jacobi_pinv(double2* A, double2* V, const double2* rhs, int s, double tol, double2* beta,
+                                 double2* coef, int* sh) {
+    const int tid = threadIdx.x;
+    const int sp = s + (s & 1);
+    for (int idx = tid; idx < sp * sp; idx += blockDim.x) {
+        const int c = idx / sp, i = idx % sp;
+        V[idx] = make_double2(c == i ? 1.0 : 0.0, 0.0);
+    }
+    __syncthreads();
+    for (int sweep = 0; sweep < 60; ++sweep) {
+        if (tid == 0) sh[0] = 0;
+        __syncthreads();
+        for (int step = 0; step < sp - 1; ++step) {
+            if (tid < sp / 2) {
+                int a, b;
+                if (tid == 0) { a = sp - 1; b = step; }
+                else { a = (step + tid) % (sp - 1); b = (step - tid + (sp - 1)) % (sp - 1); }
+                const int p = a < b ? a : b, q = a < b ? b : a;
+                double2* ap = A + p * sp;
+                double2* aq = A + q * sp;
+                double alpha = 0.0, bet = 0.0, gr = 0.0, gi = 0.0;
+                for (int i = 0; i < s; ++i) {
+                    const double2 x = ap[i], y = aq[i];
+                    alpha += x.x * x.x + x.y * x.y;
+                    bet += y.x * y.x + y.y * y.y;
+                    gr += x.x * y.x + x.y * y.y;          // conj(x) * y
+                    gi += x.x * y.y - x.y * y.x;
+                }
+                const double g2 = gr * gr + gi * gi;
+                if (g2 > 1e-30 * alpha * bet && g2 > 0.0) {
+                    const double g = sqrt(g2);
+                    const double2 ph = make_double2(gr / g, -gi / g);      // exp(-i arg gamma)
+                    const double zeta = (bet - alpha) / (2.0 * g);
+                    const double tt = copysign(1.0, zeta) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+                    const double c = 1.0 / sqrt(1.0 + tt * tt), sn = c * tt;
+                    for (int i = 0; i < s; ++i) {
+                        const double2 x = ap[i], y = cmul(aq[i], ph);
+                        ap[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
+                        aq[i] = make_double2(sn * x.x + c * y.x, sn * x.y + c * y.y);
+                    }
+                    double2* vp = V + p * sp;
+                    double2* vq = V + q * sp;
+                    for (int i = 0; i < sp; ++i) {
+                        const double2 x = vp[i], y = cmul(vq[i], ph);
+                        vp[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
+                        vq[i] = make_double2(sn * x.x + c * y.x, sn * x.y + c * y.y);
+                    }
+                    sh[0] = 1;
+                }
+            }
+            __syncthreads();
+        }
+        const int rotated = sh[0];
+        __syncthreads();
+        if (!rotated) break;
+    }
+    if (tid == 0) sh[1] = 0;
+    __syncthreads();
+    if (tid < sp) {
+        const double2* ak = A + tid * sp;
+        double sig2 = 0.0, pr = 0.0, pi = 0.0;
+        for (int i = 0; i < s; ++i) {
+            const double2 x = ak[i], r = rhs[i];
+            sig2 += x.x * x.x + x.y * x.y;
+            pr += x.x * r.x + x.y * r.y;                  // conj(x) * r
+            pi += x.x * r.y - x.y * r.x;
+        }
+        const bool keep = sqrt(sig2) > tol;
+        coef[tid] = keep ? make_double2(pr / sig2, pi / sig2) : make_double2(0.0, 0.0);
+        if (keep) atomicAdd(&sh[1], 1);
+    }
+    __syncthreads();
+    if (tid < s) {
+        double re = 0.0, im = 0.0;
+        for (int k = 0; k < sp; ++k) {
+            const double2 q = cmul(V[k * sp + tid], coef[k]);
+            re += q.x;
+            im += q.y;
+        }
+        beta[tid] = make_double2(re, im);
+    }
+    __syncthreads();
+    return sh[1];
+}
+
+// ------------------------------------------------------------------ locator after the projection
+__global__ void __launch_bounds__(kSolveThreads)
+cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ partial, int grid, const double2* __restrict__ e_in,
+                 int n, int s, double theta, uint8_t* flags, uint8_t* flags2, DeviceInfo* info) {
+    __shared__ double2 e[kMaxN], h[kMaxN];
+    __shared__ double mag[kMaxN], sorted[kMaxN];
+    __shared__ int sh[4], count;
+    __shared__ double scale_s, maxsyn_s;
+    const int tid = threadIdx.x;
+    const double rsn = 1.0 / sqrt((double)n);
+
+    if (tid < n) {
+        double2 v;
+        if (e_in != nullptr) {
+            v = e_in[tid];
+        } else {
+            double a = 0.0, b = 0.0;
+            for (int blk = 0; blk < grid; ++blk) {
+                const double2 p = partial[(int64_t)blk * n + tid];
+                a += p.x;
+                b += p.y;
+            }
+            v = make_double2(a, b);
+        }
+        e[tid] = v;
+        cd->e[tid] = v;
+        mag[tid] = sqrt(cabs2(v));
+        h[tid] = make_double2(0.0, 0.0);
+    }
+    if (tid == 0) count = 0;
+    __syncthreads();
+    // median of |e_j| by rank counting
+    if (tid < n) {
+        int rank = 0;
+        for (int k = 0; k < n; ++k) rank += (mag[k] < mag[tid]) || (mag[k] == mag[tid] && k < tid);
+        sorted[rank] = mag[tid];
+    }
+    __syncthreads();
+    if (tid == 0) scale_s = (n & 1) ? sorted[n / 2] : 0.5 * (sorted[n / 2 - 1] + sorted[n / 2]);
+    // syndromes h_m = n^(-1/2) sum_j e_j w^(-m j), m = n-2s .. n-1
+    if (tid < 2 * s) {
+        const int m = n - 2 * s + tid;
+        double a = 0.0, b = 0.0;
+        for (int j = 0; j < n; ++j) {
+            const double2 q = cmulc(e[j], cd->twiddle[(m * j) % n]);
+            a += q.x;
+            b += q.y;
+        }
+        h[m] = make_double2(a * rsn, b * rsn);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        double mx = 0.0;
+        for (int m = n - 2 * s; m < n; ++m) mx = fmax(mx, sqrt(cabs2(h[m])));
+        maxsyn_s = mx;
+    }
+    __syncthreads();
+    const double tol = theta * scale_s;
+    int rank = 0;
+    bool flagged = false;
+    if (s > 0) {
+        // row i: [h_{n-s-1-i} .. h_{n-2-i}] beta = h_{n-1-i}; stored by columns
+        const int sp = s + (s & 1);
+        double2* A = cd->work;
+        double2* V = cd->work + sp * sp;
+        double2* rhs = cd->vec;
+        double2* beta = cd->vec + kMaxN;
+        double2* coef = cd->vec + 2 * kMaxN;
+        for (int idx = tid; idx < sp * sp; idx += blockDim.x) {
+            const int c = idx / sp, i = idx % sp;
+            A[idx] = (c < s && i < s) ? h[n - s - 1 - i + c] : make_double2(0.0, 0.0);
+        }
+        if (tid < s) rhs[tid] = h[n - 1 - tid];
+        __syncthreads();
+        rank = block_jacobi_pinv(A, V, rhs, s, tol, beta, coef, sh);
+    }
+    if (rank > 0) {
+        double2* beta = cd->vec + kMaxN;
+        if (tid == 0) {
+            for (int l = 0; l < n - 2 * s; ++l) {
+                double a = 0.0, b = 0.0;
+                for (int u = 0; u < s; ++u) {
+                    int idx = l + u - s;
+                    if (idx < 0) idx += n;
+                    const double2 q = cmul(beta[u], h[idx]);
+                    a += q.x;
+                    b += q.y;
+                }
+                h[l] = make_double2(a, b);
+            }
+        }
+        __syncthreads();
+        if (tid < n) {
+            double a = 0.0, b = 0.0;
+            for (int m = 0; m < n; ++m) {
+                const double2 q = cmul(h[m], cd->twiddle[(tid * m) % n]);
+                a += q.x;
+                b += q.y;
+            }
+            const double2 t = make_double2(a * rsn, b * rsn);
+            cd->t[tid] = t;
+            mag[tid] = cabs2(t);
+        }
+        __syncthreads();
+        // exactly `rank` entries of t are non-zero in exact arithmetic: V = the rank largest |t_j|
+        if (tid < n) {
+            int pos = 0;
+            for (int k = 0; k < n; ++k) pos += (mag[k] > mag[tid]) || (mag[k] == mag[tid] && k < tid);
+            flagged = pos < rank;
+        }
+    } else if (tid < n) {
+        cd->t[tid] = make_double2(0.0, 0.0);
+    }
+    if (tid < n) {
+        cd->h[tid] = h[tid];
+        if (flags) flags[tid] = flagged ? 1 : 0;
+        if (flags2) flags2[tid] = flagged ? 1 : 0;
+        if (flagged) atomicAdd(&count, 1);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        info->n_flagged = count;
+        info->locator_rank = rank;
+        info->scale = scale_s;
+        info->max_syndrome = maxsyn_s;
+        info->status = DRACO_OK;
+        info->no_majority = 0;
+    }
+}
+
+// ------------------------------------------------------------------ decode vector
+// With B = [C_L]_{.,V} and A = [C_L]_{.,U}: A A^H = I - B B^H, so the minimum-norm solution of
+// A b_U = e_last is b_U = A^H y, y = e_last + B (I - B^H B)^{-1} B^H e_last, and
+// I - B^H B = [C_R]_{.,V}^H [C_R]_{.,V} is only |V| x |V| (|V| <= 2 s).
+__global__ void __launch_bounds__(kSolveThreads)
+cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n, int s, DeviceInfo* info) {
+    __shared__ int vlist[kMaxN], rowbestc[kMaxN], sh[4], a_s;
+    __shared__ double rowbest[kMaxN];
+    __shared__ double2 y[kMaxN];
+    const int tid = threadIdx.x;
+    const int rows = n - 2 * s, L = rows - 1;
+    const double rsn = 1.0 / sqrt((double)n);
+    if (tid == 0) {
+        int a = 0;
+        for (int j = 0; j < n; ++j)
+            if (flags[j]) vlist[a++] = j;
+        a_s = a;
+    }
+    __syncthreads();
+    const int a = a_s;
+    if (a > 2 * s) {                                       // fewer than n - 2 s rows left: no b exists
+        if (tid < n) cd->b[tid] = make_double2(0.0, 0.0);
+        if (tid == 0) { info->n_active = 0; info->n_flagged = a; info->status = DRACO_ETOOMANY; }
+        return;
+    }
+    double2* x = cd->vec;
+    if (a > 0) {
+        double2* A = cd->work;
+        for (int idx = tid; idx < a * (a + 1); idx += blockDim.x) {
+            const int p = idx / (a + 1), q = idx % (a + 1);
+            double2 val;
+            if (q < a) {                                   // (1/n) sum_{m >= n-2s} w^(m (v_q - v_p))
+                int dv = vlist[q] - vlist[p];
+                if (dv < 0) dv += n;
+                double re = 0.0, im = 0.0;
+                for (int m = n - 2 * s; m < n; ++m) {
+                    const double2 w = cd->twiddle[(m * dv) % n];
+                    re += w.x;
+                    im += w.y;
+                }
+                val = make_double2(re / n, im / n);
+            } else {                                       // conj(C[L][v_p])
+                const double2 w = cd->twiddle[(L * vlist[p]) % n];
+                val = make_double2(w.x * rsn, -w.y * rsn);
+            }
+            A[idx] = val;
+        }
+        __syncthreads();
+        block_gauss_jordan(A, a, 0.0, x, cd->perm, rowbest, rowbestc, sh);
+    }
+    if (tid < rows) {
+        double re = (tid == L) ? 1.0 : 0.0, im = 0.0;
+        for (int p = 0; p < a; ++p) {
+            const double2 w = cd->twiddle[(tid * vlist[p]) % n];
+            const double2 q = cmul(w, x[p]);
+            re += q.x * rsn;
+            im += q.y * rsn;
+        }
+        y[tid] = make_double2(re, im);
+    }
+    __syncthreads();
+    if (tid < n) {
+        double2 b = make_double2(0.0, 0.0);
+        if (!flags[tid]) {
+            double re = 0.0, im = 0.0;
+            for (int m = 0; m < rows; ++m) {
+                const double2 q = cmulc(y[m], cd->twiddle[(m * tid) % n]);
+                re += q.x;
+                im += q.y;
+            }
+            b = make_double2(re * rsn, im * rsn);
+        }
+        cd->b[tid] = b;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int k = 0;
+        for (int j = 0; j < n; ++j)
+            if (!flags[j]) {
+                cd->active[k] = j;
+                cd->b_active[k] = cd->b[j];
+                ++k;
+            }
+        info->n_active = k;
+        info->n_flagged = a;
+        if (info->status == DRACO_ETOOMANY) info->status = DRACO_OK;
+    }
+}
+
+}  // namespace
+
+int project_grid_size(int sm_count) { return sm_count * 2; }
+
+int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t len, int64_t ld, bool accumulate,
+                       cudaStream_t st) {
+    const int grid = p->project_grid;
+    const bool vec2 = (ld % 2 == 0);
+    const int n = p->n;
+#define DRACO_PROJ(RPW, V2) \
+    cyc_project_kernel<RPW, V2><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0)
+    if (vec2) {
+        if (n <= 32) DRACO_PROJ(4, true);
+        else if (n <= 64) DRACO_PROJ(8, true);
+        else DRACO_PROJ(16, true);
+    } else {
+        if (n <= 32) DRACO_PROJ(4, false);
+        else if (n <= 64) DRACO_PROJ(8, false);
+        else DRACO_PROJ(16, false);
+    }
+#undef DRACO_PROJ
+    DRACO_CUDA(cudaGetLastError());
+    return DRACO_OK;
+}
+
+int launch_cyc_project_finish(draco_plan* p, double2* e_out, cudaStream_t st) {
+    cyc_project_finish_kernel<<<1, kMaxN, 0, st>>>(p->partial_dev, p->project_grid, p->n, e_out);
+    DRACO_CUDA(cudaGetLastError());
+    return DRACO_OK;
+}
+
+int launch_cyc_solve(draco_plan* p, const double2* e, uint8_t* flags, cudaStream_t st) {
+    cyc_solve_kernel<<<1, kSolveThreads, 0, st>>>(p->cyc_dev, p->partial_dev, p->project_grid, e, p->n, p->s, p->theta,
+                                                  flags, p->flags_dev, p->info_dev);
+    DRACO_CUDA(cudaGetLastError());
+    return DRACO_OK;
+}
+
+int launch_cyc_decode_vector(draco_plan* p, const uint8_t* flags, cudaStream_t st) {
+    cyc_decode_vector_kernel<<<1, kSolveThreads, 0, st>>>(p->cyc_dev, flags, p->n, p->s, p->info_dev);
+    DRACO_CUDA(cudaGetLastError());
+    return DRACO_OK;
+}
+
+}  // namespace draco

@@ -1,0 +1,114 @@
+// Internal declarations shared by the translation units of libdraco.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "draco.h"
+
+namespace draco {
+
+constexpr int kMaxN = DRACO_MAX_N;
+constexpr int kMaxTaps = 15;          // 2 s + 1 for the register-window encoder (s <= 7)
+constexpr int kProjectTile = 2048;    // coordinates per tile of the projection kernel
+constexpr int kProjectWarps = 8;
+
+struct GroupTable {                   // repetition code: consecutive groups
+    int num_groups;
+    int max_size;
+    uint8_t first[kMaxN];
+    uint8_t size[kMaxN];
+};
+
+struct EncodeTaps {                   // cyclic encoder: z_j = phase[j] * sum_t tap[t] * g_{(j-t) mod n}
+    float2 tap[kMaxTaps];
+};
+
+struct EncodePhase {
+    float2 phase[kMaxN];
+};
+
+// Device-resident state of the cyclic decoder (lives in the plan's scratch).
+struct CycDevice {
+    double2 twiddle[kMaxN];           // w^k, w = exp(2 pi i / n)
+    double2 e[kMaxN];                 // projection f R
+    double2 h[kMaxN];                 // syndromes, then the full DFT of gamma
+    double2 t[kMaxN];                 // IDFT(h)
+    double2 b[kMaxN];                 // decode vector (zero on flagged nodes)
+    double2 b_active[kMaxN];          // b_j of the active rows, packed
+    int32_t active[kMaxN];            // their node indices
+    double2 work[kMaxN * (kMaxN + 1)];  // elimination work space
+    double2 vec[4 * kMaxN];
+    int32_t perm[kMaxN];
+};
+
+struct DeviceInfo {                   // mirrors draco_info
+    int32_t status;
+    int32_t n_flagged;
+    int32_t locator_rank;
+    int32_t n_active;
+    unsigned long long no_majority;
+    double scale;
+    double max_syndrome;
+};
+
+}  // namespace draco
+
+struct draco_plan {
+    int n, s, code;
+    int64_t d;
+    int device;
+    int sm_count;
+    double theta;
+    // repetition
+    draco::GroupTable groups;
+    // cyclic (host copies)
+    double* W_host;                   // [n][n][2]
+    draco::EncodeTaps taps;
+    draco::EncodePhase phase;
+    float2* taps_full_dev;            // generic encoder: taps for any s, device [2s+1]
+    // device scratch
+    draco::CycDevice* cyc_dev;
+    draco::DeviceInfo* info_dev;
+    double2* partial_dev;             // [project_grid][n]
+    int project_grid;
+    uint8_t* flags_dev;               // [n] internal flags
+    uint32_t* mask_dev;               // repetition: disagreement bits, [n] words
+    // host-buffer pipeline (allocated on its first call)
+    float* stage_dev;                 // [n][stage_chunk] slice of G
+    int64_t stage_chunk;
+    float* f_dev;                     // [d]
+    float* u_dev;                     // [d]
+};
+
+namespace draco {
+
+// Set the thread's last CUDA error text; returns DRACO_ECUDA.
+int cuda_fail(cudaError_t err, const char* what);
+
+#define DRACO_CUDA(call)                                              \
+    do {                                                              \
+        cudaError_t err__ = (call);                                   \
+        if (err__ != cudaSuccess) return draco::cuda_fail(err__, #call); \
+    } while (0)
+
+// kernels / launchers (one per translation unit)
+int launch_rep_encode(const draco_plan* p, const float* G, float* Z, int64_t len, int64_t ldg, int64_t ldz,
+                      cudaStream_t st);
+int launch_rep_vote(draco_plan* p, const float* R, int64_t len, int64_t ld, float* u, float* maj, uint8_t* flags,
+                    bool reset, cudaStream_t st);
+int launch_cyc_encode(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz,
+                      cudaStream_t st);
+int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t len, int64_t ld, bool accumulate,
+                       cudaStream_t st);
+int launch_cyc_project_finish(draco_plan* p, double2* e_out, cudaStream_t st);
+int launch_cyc_solve(draco_plan* p, const double2* e, uint8_t* flags, cudaStream_t st);
+int launch_cyc_decode_vector(draco_plan* p, const uint8_t* flags, cudaStream_t st);
+int launch_cyc_recover(draco_plan* p, const float2* R, int64_t len, int64_t ld, float* u, cudaStream_t st);
+int launch_generate(float* out, int rows, int64_t len, int64_t ld, int64_t i0, int row0, float mean, float std,
+                    uint64_t seed, cudaStream_t st);
+int launch_corrupt_row(float* row, int64_t nvals, int64_t v0, int model, float param, uint64_t seed, int node,
+                       bool is_complex, cudaStream_t st);
+int project_grid_size(int sm_count);
+
+}  // namespace draco

@@ -1,0 +1,284 @@
+"""Cyclic code: CUDA path vs the CPU oracle.
+
+Bars (max |a - b| / max |b| unless said otherwise):
+  W table                 <= 1e-12 of max |W|
+  encode                  <= 1e-6 per worker vector (fp32 FMA chains of 2 s + 1 terms)
+  projection e = f R      <= 1e-6 (fp32 products, fp64 sums)
+  flags, locator rank     exact
+  decode vector b         <= 1e-9
+  decode on identical R, identical flags   <= 1e-4 (the stated tolerance; observed ~1e-7)
+  end to end vs the exact sum   <= 1e-4 at (15, 2); at (45, 5) complex64 transport limits any
+                          implementation to ~1e-3, so the bar there is 2 x the oracle's own error.
+"""
+import numpy as np
+import pytest
+import torch
+
+import draco_inputs as di
+from gpu_util import dev, host, normwise
+from oracle import draco_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+# (n, s, d): config-1-like; several tiles + ragged tail; 4 does not divide d (generic encoder,
+# scalar projection / recovery); d odd; d below one tile; n = 2 s + 1; s = 0; larger s paths
+SHAPES = [(15, 2, 100_000), (45, 5, 20_484), (45, 3, 6150), (15, 2, 4098), (15, 2, 1001), (9, 1, 5), (5, 2, 300),
+          (6, 0, 516), (15, 7, 2048), (21, 4, 4100), (33, 6, 2052), (20, 8, 1028)]
+
+
+def _plan(n, s, d):
+    import paper_1803_09877_b200 as dr
+    return dr, dr.Plan(n, s, d, dr.CYC)
+
+
+@pytest.mark.parametrize("n,s", [(4, 1), (15, 2), (45, 3), (45, 5), (15, 7), (105, 7), (20, 8)])
+def test_W_table(n, s):
+    dr, plan = _plan(n, s, 8)
+    W, Wo = plan.cyc_W(), orc.cyc_W(n, s)
+    assert np.abs(W - Wo).max() <= 1e-12 * np.abs(Wo).max()
+
+
+@pytest.mark.parametrize("n,s,d", SHAPES)
+def test_encode_parity(n, s, d):
+    dr, plan = _plan(n, s, d)
+    G = di.gradient_rows(0xD2AC0 + n + s, n, d)
+    Z = torch.empty((n, 2 * d), dtype=torch.float32, device="cuda")
+    plan.encode(dev(G), Z)
+    torch.cuda.synchronize()
+    Zg = host(Z, complex64=True)
+    Zo = orc.cyc_encode(G, n, s, dtype=np.complex128)
+    for j in range(n):
+        assert np.abs(Zg[j] - Zo[j]).max() <= 1e-6 * np.abs(Zo[j]).max(), j
+
+
+def _received(n, s, d, seed, n_adv, model=di.ADV_REVGRAD, param=100.0):
+    G = di.gradient_rows(seed, n, d)
+    R = orc.cyc_encode(G, n, s)                            # complex64 worker vectors
+    adv = di.choose_adversaries(seed + 1, n, n_adv)
+    if model == di.ADV_GAUSS:
+        param = param * float(np.abs(R).max()) / 1e3      # noise far above the vectors' own scale
+    di.apply_adversaries(R, adv, [model] * n_adv, [param] * n_adv, seed=seed + 2)
+    return G, R, adv, di.projection_vector(seed + 3, d)
+
+
+@pytest.mark.parametrize("n,s,d", SHAPES)
+@pytest.mark.parametrize("n_adv_mode", ["s", "fewer", "none"])
+def test_locate_and_decode_parity_on_identical_R(n, s, d, n_adv_mode):
+    dr, plan = _plan(n, s, d)
+    n_adv = {"s": s, "fewer": max(s - 1, 0) if s < 3 else s - 2, "none": 0}[n_adv_mode]
+    model = di.ADV_GAUSS if (n + s) % 2 else di.ADV_REVGRAD
+    G, R, adv, f = _received(n, s, d, 17 * n + s, n_adv, model, 1e3 if model == di.ADV_GAUSS else 100.0)
+    want = orc.cyc_locate(R, f, n, s)
+    Rd, fd = dev(R), dev(f)
+    # projection
+    e = torch.empty(2 * n, dtype=torch.float64, device="cuda")
+    plan.cyc_project(Rd, fd, e)
+    eg = host(e).view(np.complex128)
+    assert np.abs(eg - want["e"]).max() <= 1e-6 * np.abs(want["e"]).max()
+    # locator
+    flags = torch.full((n,), 9, dtype=torch.uint8, device="cuda")
+    plan.locate(Rd, fd, flags)
+    info = plan.info()
+    fg = host(flags).astype(bool)
+    tol = 1e-6 * want["scale"]
+    sv = want.get("sv", np.zeros(0))
+    assert all(x > 3 * tol or x < tol / 3 for x in sv), "test input sits too close to the rank cutoff"
+    assert want["margin"] > 10, "test input: |t| of flagged and unflagged nodes too close"
+    np.testing.assert_array_equal(fg, want["flags"])
+    assert sorted(np.flatnonzero(fg)) == adv.tolist()
+    assert info["locator_rank"] == want["rank"] == n_adv and info["n_flagged"] == n_adv
+    assert abs(info["scale"] - want["scale"]) <= 1e-6 * want["scale"]
+    # split entry points agree with the fused one
+    flags2 = torch.empty_like(flags)
+    plan.cyc_locate_from_projection(e, flags2)
+    torch.cuda.synchronize()
+    assert torch.equal(flags, flags2)
+    # decode with the same flags on the same R
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.decode(Rd, flags, u)
+    info = plan.info()
+    assert info["status"] == 0 and info["n_active"] == n - n_adv
+    b = plan.cyc_decode_vector()
+    bo = orc.cyc_decode_vector(n, s, want["flags"])
+    assert np.abs(b - bo).max() <= 1e-9 * np.abs(bo).max()
+    uo = orc.cyc_decode(R, n, s, want["flags"])
+    assert normwise(host(u), uo) <= 1e-4
+    assert normwise(host(u), uo) <= 1e-6                    # what fp64 accumulation actually delivers
+    u2 = torch.empty_like(u)
+    f2 = torch.empty_like(flags)
+    plan.locate_decode(Rd, fd, f2, u2)
+    torch.cuda.synchronize()
+    assert torch.equal(u2, u) and torch.equal(f2, flags)
+
+
+@pytest.mark.parametrize("n,s,d,bar", [(15, 2, 100_000, 1e-4), (15, 1, 30_000, 1e-4), (45, 5, 30_000, None),
+                                        (45, 3, 30_000, None)])
+def test_pipeline_against_exact_sum(n, s, d, bar):
+    """encode -> corrupt -> locate -> decode, all on the device, against G 1_P."""
+    dr, plan = _plan(n, s, d)
+    seed = 900 + n + s
+    G = di.gradient_rows(seed, n, d)
+    adv = di.choose_adversaries(seed + 1, n, s)
+    f = di.projection_vector(seed + 3, d)
+    Gd, fd = dev(G), dev(f)
+    Z = torch.empty((n, 2 * d), dtype=torch.float32, device="cuda")
+    plan.encode(Gd, Z)
+    plan.corrupt(Z, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.locate_decode(Z, fd, flags, u)
+    torch.cuda.synchronize()
+    assert sorted(np.flatnonzero(host(flags))) == adv.tolist()
+    exact = G.astype(np.float64).sum(axis=0)
+    err = normwise(host(u), exact)
+    # the oracle's own end-to-end error with complex64 worker vectors
+    Ro = orc.cyc_encode(G, n, s)
+    di.apply_adversaries(Ro, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2)
+    out = orc.cyc_decode_full(Ro, f, n, s)
+    assert sorted(np.flatnonzero(out["flags"])) == adv.tolist()
+    floor = normwise(out["u"], exact)
+    if bar is not None:
+        assert err <= bar and floor <= bar
+    else:
+        assert err <= 2.0 * floor + 1e-6, (err, floor)
+    assert np.abs(host(u)).max() > 0
+
+
+def test_too_many_flags_is_refused_with_zero_output():
+    n, s, d = 15, 2, 2048
+    dr, plan = _plan(n, s, d)
+    R = di.complex_rows(3, n, d)
+    flags = np.zeros(n, dtype=np.uint8)
+    flags[: 2 * s + 1] = 1
+    u = torch.full((d,), 5.0, dtype=torch.float32, device="cuda")
+    plan.decode(dev(R), dev(flags), u)
+    info = plan.info()
+    assert info["status"] == dr.binding.ETOOMANY and info["n_active"] == 0
+    assert float(u.abs().max()) == 0.0
+    # 2 s flagged (erasure decoding) still works on any R: u = Re(b^T R)
+    flags[2 * s] = 0
+    plan.decode(dev(R), dev(flags), u)
+    assert plan.info()["status"] == 0
+    uo = orc.cyc_decode(R, n, s, flags.astype(bool))
+    assert normwise(host(u), uo) <= 1e-6
+
+
+def test_beyond_s_fails_visibly():
+    """s + 1 adversaries: the decoder cannot return the true sum (Theorem 1)."""
+    n, s, d = 15, 2, 8192
+    dr, plan = _plan(n, s, d)
+    G = di.gradient_rows(11, n, d)
+    R = orc.cyc_encode(G, n, s)
+    adv = [1, 6, 12]
+    di.apply_adversaries(R, adv, [di.ADV_REVGRAD] * 3, [100.0] * 3, seed=0)
+    f = di.projection_vector(12, d)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.locate_decode(dev(R), dev(f), flags, u)
+    info = plan.info()
+    wrong_set = sorted(np.flatnonzero(host(flags))) != adv
+    wrong_sum = normwise(host(u), G.astype(np.float64).sum(axis=0)) > 1e-3
+    assert wrong_set or wrong_sum or info["status"] != 0
+
+
+def test_host_pipeline_matches_device_pipeline():
+    n, s, d = 15, 2, 300_000
+    dr, plan = _plan(n, s, d)
+    seed = 4242
+    G = di.gradient_rows(seed, n, d)
+    f = di.projection_vector(seed + 3, d)
+    adv = di.choose_adversaries(seed + 1, n, s)
+    Z = torch.empty((n, 2 * d), dtype=torch.float32, device="cuda")
+    u_host = np.empty(d, dtype=np.float32)
+    flags_host = np.empty(n, dtype=np.uint8)
+    info = plan.pipeline_host(G.ctypes.data, f.ctypes.data, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed + 2, Z,
+                              u_host.ctypes.data, flags_host.ctypes.data)
+    assert info["status"] == 0 and sorted(np.flatnonzero(flags_host)) == adv.tolist()
+    assert normwise(u_host, G.astype(np.float64).sum(axis=0)) <= 1e-4
+    Z2 = torch.empty_like(Z)
+    plan.encode(dev(G), Z2)
+    plan.corrupt(Z2, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.locate_decode(Z2, dev(f), flags, u)
+    torch.cuda.synchronize()
+    assert torch.equal(Z, Z2)
+    np.testing.assert_array_equal(host(u), u_host)
+
+
+def test_full_size_resnet152_config_sampled():
+    """n = 45, s = 5, d = 60.2 M (21.7 GB of complex64 worker vectors), reversed-gradient
+    adversaries at random positions; inputs generated on the device, outputs checked on a
+    coordinate sample, the projection on sampled rows over all d."""
+    import paper_1803_09877_b200 as dr
+    n, s, d = 45, 5, 60_200_000
+    plan = dr.Plan(n, s, d, dr.CYC)
+    seed = 0xD2AC0 + 4
+    G = torch.empty((n, d), dtype=torch.float32, device="cuda")
+    dr.generate(G, n, d, seed=seed)
+    f = torch.empty(d, dtype=torch.float32, device="cuda")
+    dr.generate(f, 1, d, mean=1.0, std=1.0, seed=seed + 3)
+    Z = torch.empty((n, 2 * d), dtype=torch.float32, device="cuda")
+    plan.encode(G, Z)
+    adv = di.choose_adversaries(seed + 1, n, s)
+    plan.corrupt(Z, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.locate_decode(Z, f, flags, u)
+    info = plan.info()
+    assert sorted(np.flatnonzero(host(flags))) == adv.tolist()            # Lemma 4: V = the corrupted nodes
+    assert info["locator_rank"] == s and info["status"] == 0
+    rng = np.random.default_rng(2)
+    idx = np.unique(np.concatenate([np.arange(4096), np.arange(d - 4096, d), rng.integers(0, d, 100_000)]))
+    Gs = di.gradient_rows(seed, n, d, idx=idx)
+    np.testing.assert_array_equal(host(G[:, idx]), Gs)                     # same inputs on both sides
+    # encode on the sample
+    Zo = orc.cyc_encode(Gs, n, s, dtype=np.complex128)
+    Zg = host(Z.view(n, d, 2)[:, idx, :].contiguous().view(n, -1), complex64=True)
+    honest = np.setdiff1d(np.arange(n), adv)
+    for j in honest:
+        assert np.abs(Zg[j] - Zo[j]).max() <= 1e-6 * np.abs(Zo[j]).max()
+    # decode on the sample: identical R (the device's rows), identical flags
+    want_flags = np.zeros(n, dtype=bool)
+    want_flags[adv] = True
+    Ro = Zo.astype(np.complex64)
+    di.apply_adversaries(Ro, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2, idx=idx)
+    exact = Gs.astype(np.float64).sum(axis=0)
+    floor = normwise(orc.cyc_decode(Ro, n, s, want_flags), exact)
+    err = normwise(host(u[idx]), exact)
+    assert err <= 2.0 * floor + 1e-6, (err, floor)
+    # projection of two honest rows over all d, by the oracle's definition in chunks
+    e = torch.empty(2 * n, dtype=torch.float64, device="cuda")
+    plan.cyc_project(Z, f, e)
+    eg = host(e).view(np.complex128)
+    W = orc.cyc_W(n, s)
+    for j in (int(honest[0]), int(honest[-1])):
+        acc = 0.0 + 0.0j
+        step = 4_000_000
+        for c0 in range(0, d, step):
+            c1 = min(d, c0 + step)
+            Gc = di.gradient_rows(seed, n, d, i0=c0, i1=c1)
+            fc = di.projection_vector(seed + 3, d, i0=c0, i1=c1)
+            zj = (W[:, j] @ Gc.astype(np.complex128)).astype(np.complex64)
+            acc += orc.cyc_project(zj[None, :], fc)[0]
+        assert abs(eg[j] - acc) <= 1e-5 * abs(acc), (j, eg[j], acc)
+
+
+def test_full_size_decode_on_generated_R_sampled():
+    """Recovery kernel alone at full size on a synthetic complex64 matrix that both sides can
+    generate: identical R, identical flags, sampled coordinates."""
+    import paper_1803_09877_b200 as dr
+    n, s, d = 45, 5, 60_200_000
+    plan = dr.Plan(n, s, d, dr.CYC)
+    R = torch.empty((n, 2 * d), dtype=torch.float32, device="cuda")
+    dr.generate(R, n, 2 * d, seed=555)
+    flags = np.zeros(n, dtype=np.uint8)
+    flags[[3, 11, 12, 30, 44]] = 1
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.decode(R, dev(flags), u)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(3)
+    idx = np.unique(np.concatenate([np.arange(2048), np.arange(d - 2048, d), rng.integers(0, d, 50_000)]))
+    Rs = di.complex_rows(555, n, d, idx=idx)
+    uo = orc.cyc_decode(Rs, n, s, flags.astype(bool))
+    assert normwise(host(u[idx]), uo) <= 1e-6

@@ -1,0 +1,46 @@
+"""The CUDA generator / corruptor produce the same bits as the numpy definition."""
+import numpy as np
+import pytest
+import torch
+
+import draco_inputs as di
+from gpu_util import dev, host
+
+pytestmark = pytest.mark.gpu
+
+
+def test_generate_matches_numpy_bit_for_bit():
+    import paper_1803_09877_b200 as dr
+    for rows, length, row0, mean, std, seed in [(3, 1000, 0, 0.0, 1.0, 1), (2, 4099, 5, 1.0, 1.0, 0xD2AC0),
+                                                (1, 17, 0, 0.25, 0.1, 2 ** 63 + 11)]:
+        out = torch.empty((rows, length), dtype=torch.float32, device="cuda")
+        dr.generate(out, rows, length, row0=row0, mean=mean, std=std, seed=seed)
+        torch.cuda.synchronize()
+        want = di.approx_normal_rows(seed, range(row0, row0 + rows), 0, length, mean, std)
+        np.testing.assert_array_equal(host(out).view(np.uint32), want.view(np.uint32))
+
+
+def test_generate_f_and_complex_views():
+    import paper_1803_09877_b200 as dr
+    d = 3000
+    f = torch.empty(d, dtype=torch.float32, device="cuda")
+    dr.generate(f, 1, d, mean=1.0, std=1.0, seed=77)
+    np.testing.assert_array_equal(host(f), di.projection_vector(77, d))
+    R = torch.empty((4, 2 * d), dtype=torch.float32, device="cuda")
+    dr.generate(R, 4, 2 * d, std=3.0, seed=78)
+    np.testing.assert_array_equal(host(R, complex64=True), di.complex_rows(78, 4, d, std=3.0))
+
+
+@pytest.mark.parametrize("code", [0, 1])
+def test_corrupt_matches_numpy(code):
+    import paper_1803_09877_b200 as dr
+    n, s, d = 9, 2, 1234
+    plan = dr.Plan(n, s, d, code)
+    R0 = di.complex_rows(5, n, d) if code == dr.CYC else di.gradient_rows(5, n, d)
+    adv, model, param = [1, 4, 8], [dr.ADV_REVGRAD, dr.ADV_CONST, dr.ADV_GAUSS], [100.0, 1e4, 1e3]
+    Rd = dev(R0)
+    plan.corrupt(Rd, adv, model, param, seed=99)
+    torch.cuda.synchronize()
+    want = di.apply_adversaries(R0.copy(), adv, model, param, seed=99)
+    got = host(Rd, complex64=(code == dr.CYC))
+    np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
