@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the Draco encode -> corrupt -> locate -> decode path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one pass of the whole path over one batch of synthetic gradients resident in HBM:
+encode all n workers' vectors, apply the adversaries, locate them, decode the sum.  The default
+workload is the ResNet-152-sized cyclic-code configuration (n = 45, s = 5, d = 60.2 M).  With
+N > 1 (torchrun, one rank per GPU) every rank holds its own d-slice of that size (weak scaling);
+the only exchange is one all-reduce of the n complex projections inside the locator.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import draco_inputs as di  # noqa: E402
+
+METRIC = "coded_gradient_throughput"
+UNIT = "GB/s"
+
+WORKLOADS = {
+    # name: (code, n, s, d, gradient std, adversary models, params)
+    "cyc_n45_s5_d60.2M": ("cyc", 45, 5, 60_200_000, 1.0, ["revgrad"], [100.0]),
+    "rep_n45_s3_d11.7M": ("rep", 45, 3, 11_700_000, 0.1, ["revgrad", "const"], [100.0, 1e4]),
+    "cyc_n15_s2_d1M": ("cyc", 15, 2, 1_000_000, 1.0, ["gauss"], [1e3]),
+    "rep_n15_s2_d100k": ("rep", 15, 2, 100_000, 1.0, ["revgrad"], [100.0]),
+}
+DEFAULT_WORKLOAD = "cyc_n45_s5_d60.2M"
+MODEL_ID = {"revgrad": di.ADV_REVGRAD, "const": di.ADV_CONST, "gauss": di.ADV_GAUSS}
+SEED = 0xD2AC0
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "MEASURED_PEAKS.json hbm_gbs (of measured)"
+    except Exception:
+        return 6650.0, "fallback 6.65 TB/s (of fallback)"
+
+
+def adversaries(workload, rank=0):
+    code, n, s, d, std, models, params = WORKLOADS[workload]
+    adv = di.choose_adversaries(SEED + 1 + 1000 * 0, n, s)          # same nodes on every rank
+    model = [MODEL_ID[models[k % len(models)]] for k in range(s)]
+    param = [params[k % len(params)] for k in range(s)]
+    return adv, model, param
+
+
+def algorithmic_bytes(code, n, s, d, n_adv):
+    """Bytes each stage must move (per step, one GPU)."""
+    if code == "cyc":
+        return {"encode": 4 * n * d + 8 * n * d, "locate": 8 * n * d + 4 * d, "decode": 8 * (n - n_adv) * d + 4 * d,
+                "corrupt": 2 * 8 * n_adv * d, "coded": 8 * n * d}
+    return {"encode": 4 * n * d + 4 * n * d, "locate": 0, "decode": 4 * n * d + 4 * d, "corrupt": 2 * 4 * n_adv * d,
+            "coded": 4 * n * d}
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def oracle_step(workload, d_sample, seed):
+    """The oracle, as it stands, on the first d_sample coordinates of the workload."""
+    from oracle import draco_oracle as orc
+    code, n, s, d, std, models, params = WORKLOADS[workload]
+    adv, model, param = adversaries(workload)
+    G = di.gradient_rows(seed, n, d, 0.0, std, i0=0, i1=d_sample)
+    f = di.projection_vector(seed + 3, d, i0=0, i1=d_sample)
+    t0 = time.perf_counter()
+    if code == "cyc":
+        R = orc.cyc_encode(G, n, s)
+        di.apply_adversaries(R, adv, model, param, seed=seed + 2)
+        out = orc.cyc_decode_full(R, f, n, s)
+        ok = sorted(np.flatnonzero(out["flags"])) == adv.tolist()
+    else:
+        R = orc.rep_encode(G, n, s)
+        di.apply_adversaries(R, adv, model, param, seed=seed + 2)
+        out = orc.rep_decode(R, n, s)
+        ok = sorted(np.flatnonzero(out["flags"])) == adv.tolist()
+    dt = time.perf_counter() - t0
+    return dt, ok
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        infos = threadpool_info()
+        return max([i.get("num_threads", 1) for i in infos] + [1])
+    except Exception:
+        return 1
+
+
+def cpu_baseline(workload, target_seconds=15.0):
+    code, n, s, d, std, models, params = WORKLOADS[workload]
+    probe = min(d, 100_000)
+    dt, _ = oracle_step(workload, probe, SEED)
+    d_sample = int(min(d, max(probe, probe * target_seconds / max(dt, 1e-3))))
+    dt, ok = oracle_step(workload, d_sample, SEED)
+    per = 8 if code == "cyc" else 4
+    return {"value": per * n * d_sample / dt / 1e9, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"first {d_sample} of {d} coordinates, all {n} workers, one pass in {dt:.2f} s "
+                      f"(numpy fp64/complex128; flags correct: {ok})"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    workload = args.workload
+    code, n, s, d, std, models, params = WORKLOADS[workload]
+    probe = min(d, 50_000)
+    dt, _ = oracle_step(workload, probe, SEED)
+    budget = 150.0 / max(1, args.steps + args.warmup)                  # seconds per step
+    d_sample = int(min(d, max(10_000, probe * min(budget, 3.0) / max(dt, 1e-3))))
+    for _ in range(args.warmup):
+        oracle_step(workload, d_sample, SEED)
+    times = []
+    for _ in range(args.steps):
+        dt, ok = oracle_step(workload, d_sample, SEED)
+        times.append(dt)
+    per = 8 if code == "cyc" else 4
+    mean = sum(times) / len(times)
+    value = per * n * d_sample / mean / 1e9
+    sample = f"first {d_sample} of {d} coordinates per step, all {n} workers (numpy fp64/complex128 oracle)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload, "code": code, "n": n, "s": s, "d": d, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- GPU arm
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.path = tempfile.mktemp(prefix="draco_clocks_", suffix=".csv")
+        self.proc = None
+        try:
+            self.fh = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.fh,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.fh.close()
+        sm, mx, reasons = [], [], set()
+        try:
+            for ln in open(self.path):
+                p = [x.strip() for x in ln.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1]))
+                    mx.append(float(p[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_1803_09877_b200 as dr
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    workload = args.workload
+    code, n, s, d, std, models, params = WORKLOADS[workload]
+    cyc = code == "cyc"
+    adv, model, param = adversaries(workload)
+    plan = dr.Plan(n, s, d, dr.CYC if cyc else dr.REP)
+    stream = torch.cuda.current_stream()
+
+    # inputs resident in HBM; rank r holds coordinates [r d, (r+1) d) of a d * world vector
+    G = torch.empty((n, d), dtype=torch.float32, device="cuda")
+    dr.generate(G, n, d, mean=0.0, std=std, seed=SEED + 17 * rank)
+    f = None
+    if cyc:
+        f = torch.empty(d, dtype=torch.float32, device="cuda")
+        dr.generate(f, 1, d, mean=1.0, std=1.0, seed=SEED + 3 + 17 * rank)
+    Z = torch.empty((n, (2 if cyc else 1) * d), dtype=torch.float32, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    e = torch.empty(2 * n, dtype=torch.float64, device="cuda")
+
+    names = ["encode", "corrupt", "locate", "decode"]
+
+    def step(ev=None):
+        def mark(i):
+            if ev is not None:
+                ev[i].record(stream)
+        mark(0)
+        plan.encode(G, Z)
+        mark(1)
+        plan.corrupt(Z, adv, model, param, seed=SEED + 2)
+        mark(2)
+        if cyc:
+            if world > 1:
+                plan.cyc_project(Z, f, e)
+                dist.all_reduce(e)
+                plan.cyc_locate_from_projection(e, flags)
+            else:
+                plan.locate(Z, f, flags)
+            mark(3)
+            plan.decode(Z, flags, u)
+        else:
+            mark(3)
+            plan.locate_decode(Z, None, flags, u)
+        mark(4)
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sync_all()
+    got = sorted(np.flatnonzero(flags.cpu().numpy()).tolist())
+    if got != adv.tolist():
+        raise SystemExit(f"flags {got} differ from the planted adversaries {adv.tolist()}")
+
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    time.sleep(0.3)
+    sync_all()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_stop = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for k in range(args.steps):
+        step(events[k])
+    t_stop.record(stream)
+    sync_all()
+    clocks = sampler.stop() if sampler else None
+    total_ms = t_start.elapsed_time(t_stop)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    stage_ms = {nm: statistics.mean(events[k][i].elapsed_time(events[k][i + 1]) for k in range(args.steps))
+                for i, nm in enumerate(names)}
+
+    ab = algorithmic_bytes(code, n, s, d, len(adv))
+    value = ab["coded"] * world / (ms_per_step * 1e-3) / 1e9
+    peak, peak_src = measured_peak_gbs()
+    if cyc:
+        dom, dom_kernel = "encode", f"cyc_encode_kernel<S={s}>"
+    else:
+        dom, dom_kernel = "decode", "rep_vote_kernel"
+    achieved = ab[dom] / (stage_ms[dom] * 1e-3) / 1e9
+    stages = {}
+    for nm in names:
+        if stage_ms[nm] > 0 and ab.get(nm, 0) > 0:
+            g = ab[nm] / (stage_ms[nm] * 1e-3) / 1e9
+            stages[nm] = {"ms": round(stage_ms[nm], 4), "algorithmic_GB": round(ab[nm] / 1e9, 4),
+                          "GB/s": round(g, 1), "frac_of_peak": round(g / peak, 4)}
+        else:
+            stages[nm] = {"ms": round(stage_ms[nm], 4)}
+    launches = (1 + len(adv) + (2 if cyc else 0) + 2 + (1 if (cyc and world > 1) else 0)) * args.steps
+
+    # end to end through the host-buffer entry point (rank-local; H2D of G and f, D2H of u and flags)
+    e2e = None
+    if not args.no_e2e:
+        del events
+        Gh = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        Gh.copy_(G)
+        fh = torch.empty(d, dtype=torch.float32, pin_memory=True)
+        if cyc:
+            fh.copy_(f)
+        uh = torch.empty(d, dtype=torch.float32, pin_memory=True)
+        flh = torch.empty(n, dtype=torch.uint8, pin_memory=True)
+        torch.cuda.synchronize()
+        reps = max(2, min(args.steps, 5))
+        plan.pipeline_host(Gh, fh if cyc else None, adv, model, param, SEED + 2, Z, uh, flh)   # warm-up, allocs
+        sync_all()
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            info = plan.pipeline_host(Gh, fh if cyc else None, adv, model, param, SEED + 2, Z, uh, flh)
+        sync_all()
+        dt = (time.perf_counter() - t0) / reps
+        if world > 1:
+            t = torch.tensor([dt], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        if sorted(np.flatnonzero(flh.numpy()).tolist()) != adv.tolist():
+            raise SystemExit("host pipeline: flags differ from the planted adversaries")
+        e2e = {"value": ab["coded"] * world / dt / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": 4 * n * d + (4 * d if cyc else 0), "d2h_bytes_per_step": 4 * d + n,
+               "ms_per_step": dt * 1e3, "steps": reps}
+
+    if rank == 0:
+        cb = cpu_baseline(workload) if (world == 1 and not args.no_cpu_baseline) else None
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32 (complex64 vectors; f64 accumulation in locate/decode)"
+                if cyc else "f32 (u32 bit patterns in the vote)", "data": "synthetic",
+                "config": {"workload": workload, "code": code, "n": n, "s": s, "d_per_gpu": d, "adversaries": len(adv),
+                           "adversary_models": models, "l2": "inputs larger than L2 (no flush needed)"
+                           if ab["coded"] > 4e8 else "working set near L2 size: not an HBM number",
+                           "value_is": "bytes of coded gradients (n d complex64 / fp32) per step / step time"},
+                "roofline": {"bound": "hbm", "kernel": dom_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                             "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                             "algorithmic_bytes_per_launch": ab[dom], "avg_launch_ms": stage_ms[dom]},
+                "stages": stages, "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "cpu_baseline": cb}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--d", type=int, default=None, help="override the workload's d (profiling on a small case)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.d is not None:
+        w = list(WORKLOADS[args.workload])
+        w[3] = args.d
+        args.workload = f"{args.workload}@d={args.d}"
+        WORKLOADS[args.workload] = tuple(w)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

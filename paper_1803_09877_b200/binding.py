@@ -11,7 +11,7 @@ import os
 
 REP, CYC = 0, 1
 ADV_REVGRAD, ADV_CONST, ADV_GAUSS = 0, 1, 2
-OK, EINVAL, ECUDA, ETOOMANY, ENOMEM, ENOMAJ = 0, -1, -2, -3, -4, 1
+OK, EINVAL, ECUDA, ETOOMANY, ENOMEM, EINTERNAL, ENOMAJ = 0, -1, -2, -3, -4, -5, 1
 MAX_N = 128
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -24,7 +24,7 @@ class DracoError(RuntimeError):
 class DracoInfo(C.Structure):
     _fields_ = [("status", C.c_int32), ("n_flagged", C.c_int32), ("locator_rank", C.c_int32),
                 ("n_active", C.c_int32), ("no_majority", C.c_uint64), ("scale", C.c_double),
-                ("max_syndrome", C.c_double)]
+                ("max_syndrome", C.c_double), ("internal_error", C.c_int32), ("reserved", C.c_int32)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}

@@ -11,135 +11,354 @@
 // rotation per output.  The taps do not depend on j, so they sit in the kernel's constant
 // parameter bank and every multiply-add takes its coefficient from there.
 //
-// A thread owns 4 consecutive coordinates and walks the n rows once, keeping a sliding
-// window of 2 s + 1 rows (plus PF rows of prefetch) in registers; the first 2 s rows of the
-// circle are fetched a second time at the end of the walk (they come from L2).
-// HBM traffic: 4 n len bytes read + 8 n len bytes written; 2 n (2 s + 1) FMA per coordinate.
+// Data movement.  A thread block owns a tile of 1024 coordinates and walks the n rows once.
+// One producer lane streams the row tiles (4 KB each) from global memory into a ring of
+// shared-memory stages with bulk asynchronous copies (cp.async.bulk + mbarrier, no
+// multicast); 8 consumer warps take each row from the ring into a register window of the
+// last 2 s + 1 rows, 4 coordinates per thread.  The first 2 s rows are also kept in shared
+// memory, because the circle closes on them at the end of the walk; nothing is read twice.
+// HBM traffic is the algorithmic minimum: 4 n len bytes read + 8 n len bytes written.
+//
+// Arithmetic.  |tap| peaks in the middle of the filter (1.8e5 at n = 45, s = 5) and decoding
+// cancels the sum back to O(1), so rounding in the encoder is amplified by that factor.  The
+// outer taps are accumulated in fp32, smallest first; the three centre taps, the rotation
+// and the final sum run in fp64, and each output is rounded to fp32 once.  That keeps the
+// encoder at the accuracy floor of complex64 transport (2 n (2 s + 1) FMA per coordinate,
+// of which 6 n + 4 n in fp64).
 #include "draco_internal.cuh"
 
 namespace draco {
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kConsumers = 256;                 // consumer threads (8 warps); warp 8 is the producer
+constexpr int kRingThreads = kConsumers + 32;
+constexpr int kVec = 4;                         // coordinates per consumer thread
+constexpr int kTile = kConsumers * kVec;        // coordinates per tile = floats per stage
+constexpr int kStages = 16;                     // ring depth (64 KB in flight per block)
+constexpr int kGenericThreads = 256;
 
-template <int S, int PF>
-__global__ void __launch_bounds__(kThreads, 2)
-cyc_encode_kernel(const float* __restrict__ G, float2* __restrict__ Z, int64_t len, int64_t ldg, int64_t ldz, int n,
-                  const __grid_constant__ EncodeTaps taps, const __grid_constant__ EncodePhase ph) {
-    constexpr int R = 2 * S + 1;
-    constexpr int SLOTS = R + PF;
-    const int total = n + 2 * S;          // virtual rows: the last 2 s rows of the circle, then rows 0 .. n-1
-    const int64_t nvec = len / 4;
-    const int64_t stride = (int64_t)gridDim.x * kThreads;
-    for (int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x; v < nvec; v += stride) {
-        const float* gcol = G + v * 4;
-        float2* zcol = Z + v * 4;
-        float4 win[SLOTS];
+// ---------------------------------------------------------------- mbarrier / bulk-copy wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t a, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(a), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t a, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(a), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t a, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(a), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: every wait in this file gives up after about 4 M polls (seconds), so a
+// protocol error ends the kernel with an error flag instead of hanging the device.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t a, uint32_t parity) {
+    for (int i = 0; i < (1 << 22); ++i)
+        if (mbar_try_wait(a, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity) {
+    if (mbar_try_wait(a, parity)) return true;
+    return mbar_wait_slow(a, parity);
+}
+// Hand a ring stage back to the producer after its contents were read into registers with
+// value bits `bits`.  The arrival count is 1 + ((bits * bits + bits) & 1) = 1 (x (x + 1) is
+// even), written so that the instruction carries a true register dependency on the loaded
+// data: the stage cannot be returned to the copy engine (which overwrites it through the
+// asynchronous proxy) before the shared-memory read that produced `bits` has completed.
+// Releasing straight after issuing the read lost that race under load.
+__device__ __forceinline__ void mbar_release_after_read(uint32_t a, uint32_t bits) {
+    const uint32_t count = 1u + ((bits * bits + bits) & 1u);
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(a), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t mbar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(mbar)
+                 : "memory");
+}
+
+// ---------------------------------------------------------------- consumer state
+template <int S>
+struct Window {
+    static constexpr int R = 2 * S + 1;
+    static constexpr int NBIG = R < 3 ? R : 3;                     // centre taps in fp64
+    static constexpr int H = (NBIG - 1) / 2;
+    static constexpr int SL = ((R + NBIG - 1) / NBIG) * NBIG;      // register slots: a multiple of NBIG
+    float4 win[SL];                                                // rows (vv - t), slot = vv mod SL
+    double cw[NBIG][4];                                            // fp64 copies of the rows under the centre taps
+};
+
+struct RingState {
+    uint32_t full0, empty0;      // shared addresses of the barrier arrays
+    uint32_t st, par;            // next stage to consume and its phase parity
+    uint32_t pend_bar, pend_bits;
+    bool pending;                // a stage was read in the previous step and is not released yet
+};
+
+// One step of the walk: bring row vv of the tile into window slot P (from the ring, or from
+// the stash once the circle has closed), and emit z_{vv mod n} when the window is full.
+// MODE 0: first SL steps of a tile (all rows from the ring; outputs from step 2 S on; nothing
+//         pending at step 0);  MODE 1: steady state (ring row + output, previous stage pending);
+// MODE 2: anything (run-time guards).  Returns false when a wait gave up.
+template <int S, int P, int MODE>
+__device__ __forceinline__ bool encode_step(Window<S>& w, RingState& rs, int vv, int n, const float* ring_t,
+                                            float* stash_t, float2* zcol, int64_t ldz, bool active, int lane,
+                                            const EncodeTaps& taps, const EncodeTaps64& taps64,
+                                            const EncodePhase64& ph64) {
+    constexpr int R = Window<S>::R, NBIG = Window<S>::NBIG, H = Window<S>::H, SL = Window<S>::SL;
+    const int total = n + 2 * S;
+    if (MODE == 2 && vv >= total) return true;
+    const bool from_ring = (MODE != 2) || (vv < n);
+    const bool release_first = (MODE == 1) || (MODE == 0 && P > 0) || (MODE == 2 && rs.pending);
+    if (release_first) {
+        __syncwarp();
+        if (lane == 0) mbar_release_after_read(rs.pend_bar, rs.pend_bits);
+        rs.pending = false;
+    }
+    float4 x;
+    if (from_ring) {
+        const uint32_t bar = rs.full0 + 8 * rs.st;
+        if (!mbar_wait(bar, rs.par)) return false;
+        x = *reinterpret_cast<const float4*>(ring_t + rs.st * kTile);
+        rs.pend_bar = rs.empty0 + 8 * rs.st;
+        rs.pend_bits = __float_as_uint(x.x);
+        rs.pending = true;
+        rs.st = (rs.st + 1) & (kStages - 1);
+        rs.par ^= (rs.st == 0);
+        if ((MODE == 0 && P < 2 * S) || (MODE == 2 && vv < 2 * S))
+            *reinterpret_cast<float4*>(stash_t + vv * kTile) = x;
+    } else {
+        x = *reinterpret_cast<const float4*>(stash_t + (vv - n) * kTile);
+    }
+    w.win[P] = x;
+    if (MODE != 2 || vv >= S - H) {          // the row now under tap S-H enters the fp64 window
+        constexpr int Q = (P - (S - H) + 2 * SL) % SL;
+        w.cw[Q % NBIG][0] = (double)w.win[Q].x;
+        w.cw[Q % NBIG][1] = (double)w.win[Q].y;
+        w.cw[Q % NBIG][2] = (double)w.win[Q].z;
+        w.cw[Q % NBIG][3] = (double)w.win[Q].w;
+    }
+    const bool emit = (MODE == 1) || (MODE == 0 && P >= 2 * S) || (MODE == 2 && vv >= 2 * S);
+    if (emit) {
+        // win[(P - t) mod SL] = row (vv - t) mod n: this output is z_j, j = vv mod n
+        const int j = (MODE == 2 && vv >= n) ? vv - n : vv;
+        float ar[4] = {0.f, 0.f, 0.f, 0.f}, ai[4] = {0.f, 0.f, 0.f, 0.f};
+        // taps grow towards the middle of the filter: add the outer (small) terms first so the
+        // running sums stay small while most of the fp32 roundings happen
 #pragma unroll
-        for (int p = 0; p < PF; ++p) {
-            if (p < total) {
-                int r = p - 2 * S;
-                if (r < 0) r += n;
-                win[p] = __ldcs(reinterpret_cast<const float4*>(gcol + (int64_t)r * ldg));
-            }
+        for (int k = 0; k < R; ++k) {
+            const int t = (k & 1) ? 2 * S - (k >> 1) : (k >> 1);
+            if (t >= S - H && t <= S + H) continue;
+            const float4 g = w.win[(P - t + 2 * SL) % SL];
+            const float cr = taps.tap[t].x, ci = taps.tap[t].y;
+            ar[0] = fmaf(cr, g.x, ar[0]); ai[0] = fmaf(ci, g.x, ai[0]);
+            ar[1] = fmaf(cr, g.y, ar[1]); ai[1] = fmaf(ci, g.y, ai[1]);
+            ar[2] = fmaf(cr, g.z, ar[2]); ai[2] = fmaf(ci, g.z, ai[2]);
+            ar[3] = fmaf(cr, g.w, ar[3]); ai[3] = fmaf(ci, g.w, ai[3]);
         }
-        for (int v0 = 0; v0 < total; v0 += SLOTS) {
+        double dr[4], di[4];
 #pragma unroll
-            for (int p = 0; p < SLOTS; ++p) {
-                const int vv = v0 + p;
-                if (vv < total) {
-                    if (vv + PF < total) {
-                        int r = vv + PF - 2 * S;
-                        if (r < 0) r += n;
-                        win[(p + PF) % SLOTS] = __ldcs(reinterpret_cast<const float4*>(gcol + (int64_t)r * ldg));
-                    }
-                    if (vv >= 2 * S) {
-                        const int j = vv - 2 * S;
-                        float ar0 = 0.f, ar1 = 0.f, ar2 = 0.f, ar3 = 0.f;
-                        float ai0 = 0.f, ai1 = 0.f, ai2 = 0.f, ai3 = 0.f;
+        for (int c = 0; c < 4; ++c) { dr[c] = (double)ar[c]; di[c] = (double)ai[c]; }
 #pragma unroll
-                        for (int t = 0; t < R; ++t) {
-                            const float4 g = win[(p - t + 2 * SLOTS) % SLOTS];
-                            const float cr = taps.tap[t].x, ci = taps.tap[t].y;
-                            ar0 = fmaf(cr, g.x, ar0); ai0 = fmaf(ci, g.x, ai0);
-                            ar1 = fmaf(cr, g.y, ar1); ai1 = fmaf(ci, g.y, ai1);
-                            ar2 = fmaf(cr, g.z, ar2); ai2 = fmaf(ci, g.z, ai2);
-                            ar3 = fmaf(cr, g.w, ar3); ai3 = fmaf(ci, g.w, ai3);
-                        }
-                        const float2 w = ph.phase[j];
-                        float4 lo, hi;
-                        lo.x = fmaf(ar0, w.x, -ai0 * w.y); lo.y = fmaf(ar0, w.y, ai0 * w.x);
-                        lo.z = fmaf(ar1, w.x, -ai1 * w.y); lo.w = fmaf(ar1, w.y, ai1 * w.x);
-                        hi.x = fmaf(ar2, w.x, -ai2 * w.y); hi.y = fmaf(ar2, w.y, ai2 * w.x);
-                        hi.z = fmaf(ar3, w.x, -ai3 * w.y); hi.w = fmaf(ar3, w.y, ai3 * w.x);
-                        float4* dst = reinterpret_cast<float4*>(zcol + (int64_t)j * ldz);
-                        __stcs(dst, lo);
-                        __stcs(dst + 1, hi);
-                    }
+        for (int t = S - H; t <= S + H; ++t) {
+            constexpr int dummy = 0;
+            (void)dummy;
+            const int q = ((P - t + 2 * SL) % SL) % NBIG;
+            const double cr = taps64.tap[t].x, ci = taps64.tap[t].y;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { dr[c] = fma(cr, w.cw[q][c], dr[c]); di[c] = fma(ci, w.cw[q][c], di[c]); }
+        }
+        const double2 rot = ph64.phase[j];
+        float zr[4], zi[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            zr[c] = (float)fma(dr[c], rot.x, -di[c] * rot.y);
+            zi[c] = (float)fma(dr[c], rot.y, di[c] * rot.x);
+        }
+        if (active) {
+            float4* dst = reinterpret_cast<float4*>(zcol + (int64_t)j * ldz);
+            __stcs(dst, make_float4(zr[0], zi[0], zr[1], zi[1]));
+            __stcs(dst + 1, make_float4(zr[2], zi[2], zr[3], zi[3]));
+        }
+    }
+    return true;
+}
+
+template <int S, int MODE, int P = 0>
+__device__ __forceinline__ bool encode_chunk(Window<S>& w, RingState& rs, int v0, int n, const float* ring_t,
+                                             float* stash_t, float2* zcol, int64_t ldz, bool active, int lane,
+                                             const EncodeTaps& taps, const EncodeTaps64& taps64,
+                                             const EncodePhase64& ph64) {
+    if constexpr (P < Window<S>::SL) {
+        if (!encode_step<S, P, MODE>(w, rs, v0 + P, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64))
+            return false;
+        return encode_chunk<S, MODE, P + 1>(w, rs, v0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
+    } else {
+        return true;
+    }
+}
+
+template <int S>
+__global__ void __launch_bounds__(kRingThreads)
+cyc_encode_ring_kernel(const float* __restrict__ G, float2* __restrict__ Z, int64_t len, int64_t ldg, int64_t ldz, int n,
+                       const __grid_constant__ EncodeTaps taps, const __grid_constant__ EncodeTaps64 taps64,
+                       const __grid_constant__ EncodePhase64 ph64, int* err) {
+    constexpr int SL = Window<S>::SL;
+    constexpr int NSTASH = S > 0 ? 2 * S : 1;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float* ring = reinterpret_cast<float*>(smem_raw);                        // [kStages][kTile]
+    float* stash = ring + kStages * kTile;                                   // [2 S][kTile]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(stash + NSTASH * kTile);    // full[kStages], empty[kStages]
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kStages);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, kConsumers / 32);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int64_t ntiles = (len + kTile - 1) / kTile;
+
+    if (warp == kConsumers / 32) {
+        // ---------------- producer: one lane streams row tiles into the ring
+        if (lane == 0) {
+            uint32_t cnt = 0;
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+                const int64_t c0 = tile * kTile;
+                const uint32_t bytes = (uint32_t)(((len - c0) < kTile ? (len - c0) : kTile) * 4);
+                const float* src = G + c0;
+                for (int r = 0; r < n; ++r, ++cnt, src += ldg) {
+                    const uint32_t st = cnt & (kStages - 1), par = (cnt / kStages) & 1;
+                    if (!mbar_wait(empty0 + 8 * st, par ^ 1)) { ok = false; break; }
+                    mbar_expect_tx(full0 + 8 * st, bytes);
+                    bulk_g2s(smem_u32(ring + st * kTile), src, bytes, full0 + 8 * st);
                 }
             }
+            if (!ok) {
+                atomicExch(err, 1);
+                // let the copies already in flight land before the block's shared memory is released
+                for (uint32_t back = 1; back <= kStages && back <= cnt; ++back) {
+                    const uint32_t c = cnt - back;
+                    mbar_wait(full0 + 8 * (c & (kStages - 1)), (c / kStages) & 1);
+                }
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers
+    Window<S> w;
+    RingState rs;
+    rs.full0 = full0; rs.empty0 = empty0; rs.st = 0; rs.par = 0;
+    rs.pend_bar = 0; rs.pend_bits = 0; rs.pending = false;
+    const float* ring_t = ring + tid * kVec;
+    float* stash_t = stash + tid * kVec;
+    const int total = n + 2 * S;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int64_t c0 = tile * kTile;
+        const bool active = c0 + tid * kVec < len;
+        float2* zcol = Z + c0 + tid * kVec;
+        bool ok = true;
+        int v0 = 0;
+        if (n >= SL && S > 0) {
+            ok = encode_chunk<S, 0>(w, rs, 0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
+            for (v0 = SL; ok && v0 + SL <= n; v0 += SL)
+                ok = encode_chunk<S, 1>(w, rs, v0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
+        }
+        for (; ok && v0 < total; v0 += SL)
+            ok = encode_chunk<S, 2>(w, rs, v0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
+        if (!ok) {
+            atomicExch(err, 2);
+            return;
+        }
+        if (rs.pending) {                      // only when the tile ended on a ring row (s = 0)
+            __syncwarp();
+            if (lane == 0) mbar_release_after_read(rs.pend_bar, rs.pend_bits);
+            rs.pending = false;
         }
     }
 }
 
-// Any s, any length / alignment: one coordinate per thread, rows re-read through the caches.
-__global__ void __launch_bounds__(kThreads)
+// Any s, any length / alignment: one coordinate per thread, rows re-read through the caches,
+// fp64 accumulation throughout.
+__global__ void __launch_bounds__(kGenericThreads)
 cyc_encode_generic_kernel(const float* __restrict__ G, float2* __restrict__ Z, int64_t len, int64_t ldg, int64_t ldz,
-                          int n, int s,
-                          const float2* __restrict__ taps, const __grid_constant__ EncodePhase ph) {
-    const int64_t stride = (int64_t)gridDim.x * kThreads;
-    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < len; i += stride) {
+                          int n, int s, const float2* __restrict__ taps, const __grid_constant__ EncodePhase64 ph) {
+    const int64_t stride = (int64_t)gridDim.x * kGenericThreads;
+    for (int64_t i = (int64_t)blockIdx.x * kGenericThreads + threadIdx.x; i < len; i += stride) {
         for (int j = 0; j < n; ++j) {
-            float ar = 0.f, ai = 0.f;
+            double ar = 0.0, ai = 0.0;
             for (int t = 0; t <= 2 * s; ++t) {
                 int r = j - t;
                 if (r < 0) r += n;
-                const float g = G[(int64_t)r * ldg + i];
+                const double g = (double)G[(int64_t)r * ldg + i];
                 const float2 c = taps[t];
-                ar = fmaf(c.x, g, ar);
-                ai = fmaf(c.y, g, ai);
+                ar = fma((double)c.x, g, ar);
+                ai = fma((double)c.y, g, ai);
             }
-            const float2 w = ph.phase[j];
-            Z[(int64_t)j * ldz + i] = make_float2(fmaf(ar, w.x, -ai * w.y), fmaf(ar, w.y, ai * w.x));
+            const double2 rot = ph.phase[j];
+            Z[(int64_t)j * ldz + i] = make_float2((float)fma(ar, rot.x, -ai * rot.y), (float)fma(ar, rot.y, ai * rot.x));
         }
     }
 }
 
 template <int S>
-void launch_fast(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz, cudaStream_t st) {
-    constexpr int PF = 6;
-    const int64_t nvec = len / 4;
-    int64_t want = (nvec + kThreads - 1) / kThreads;
-    const int64_t cap = (int64_t)p->sm_count * 2 * 8;
-    if (want > cap) want = cap;
-    if (want < 1) want = 1;
-    cyc_encode_kernel<S, PF><<<(int)want, kThreads, 0, st>>>(G, Z, len, ldg, ldz, p->n, p->taps, p->phase);
+int launch_ring(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz, cudaStream_t st) {
+    constexpr int NSTASH = S > 0 ? 2 * S : 1;
+    const size_t smem = sizeof(float) * kTile * (kStages + NSTASH) + 16 * kStages;
+    auto kern = cyc_encode_ring_kernel<S>;
+    static bool configured[64] = {};
+    int dev = p->device;
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (!configured[dev]) {
+        DRACO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured[dev] = true;
+    }
+    int per_sm = 1;
+    DRACO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kRingThreads, smem));
+    if (per_sm < 1) per_sm = 1;
+    const int64_t ntiles = (len + kTile - 1) / kTile;
+    int64_t grid = (int64_t)p->sm_count * per_sm;
+    if (grid > ntiles) grid = ntiles;
+    if (grid < 1) grid = 1;
+    kern<<<(int)grid, kRingThreads, smem, st>>>(G, Z, len, ldg, ldz, p->n, p->taps, p->taps64, p->phase64,
+                                               &p->info_dev->internal_error);
+    DRACO_CUDA(cudaGetLastError());
+    return DRACO_OK;
 }
 
 }  // namespace
 
 int launch_cyc_encode(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz,
                       cudaStream_t st) {
+    // the ring kernel needs 16-byte aligned row tiles: every row start and tile start a multiple of 4 floats
     const bool fast = (len % 4 == 0) && (ldg % 4 == 0) && (ldz % 2 == 0) && p->s <= 7;
     if (fast) {
         switch (p->s) {
-            case 0: launch_fast<0>(p, G, Z, len, ldg, ldz, st); break;
-            case 1: launch_fast<1>(p, G, Z, len, ldg, ldz, st); break;
-            case 2: launch_fast<2>(p, G, Z, len, ldg, ldz, st); break;
-            case 3: launch_fast<3>(p, G, Z, len, ldg, ldz, st); break;
-            case 4: launch_fast<4>(p, G, Z, len, ldg, ldz, st); break;
-            case 5: launch_fast<5>(p, G, Z, len, ldg, ldz, st); break;
-            case 6: launch_fast<6>(p, G, Z, len, ldg, ldz, st); break;
-            default: launch_fast<7>(p, G, Z, len, ldg, ldz, st); break;
+            case 0: return launch_ring<0>(p, G, Z, len, ldg, ldz, st);
+            case 1: return launch_ring<1>(p, G, Z, len, ldg, ldz, st);
+            case 2: return launch_ring<2>(p, G, Z, len, ldg, ldz, st);
+            case 3: return launch_ring<3>(p, G, Z, len, ldg, ldz, st);
+            case 4: return launch_ring<4>(p, G, Z, len, ldg, ldz, st);
+            case 5: return launch_ring<5>(p, G, Z, len, ldg, ldz, st);
+            case 6: return launch_ring<6>(p, G, Z, len, ldg, ldz, st);
+            default: return launch_ring<7>(p, G, Z, len, ldg, ldz, st);
         }
-    } else {
-        int64_t want = (len + kThreads - 1) / kThreads;
-        const int64_t cap = (int64_t)p->sm_count * 16;
-        if (want > cap) want = cap;
-        if (want < 1) want = 1;
-        cyc_encode_generic_kernel<<<(int)want, kThreads, 0, st>>>(G, Z, len, ldg, ldz, p->n, p->s, p->taps_full_dev, p->phase);
     }
+    int64_t want = (len + kGenericThreads - 1) / kGenericThreads;
+    const int64_t cap = (int64_t)p->sm_count * 16;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    cyc_encode_generic_kernel<<<(int)want, kGenericThreads, 0, st>>>(G, Z, len, ldg, ldz, p->n, p->s, p->taps_full_dev,
+                                                                     p->phase64);
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }

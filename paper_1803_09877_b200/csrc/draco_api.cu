@@ -78,10 +78,15 @@ int build_cyclic_tables(draco_plan* p, std::vector<float2>* taps_full, std::vect
     }
     taps_full->resize(2 * s + 1);
     memset(&p->taps, 0, sizeof(p->taps));
+    memset(&p->taps64, 0, sizeof(p->taps64));
+    memset(&p->phase64, 0, sizeof(p->phase64));
     for (int t = 0; t <= 2 * s; ++t) {
         const cld v = root_of_unity(n, -(long long)t * M) * w0[t];
         (*taps_full)[t] = make_float2((float)v.real(), (float)v.imag());
-        if (t < kMaxTaps) p->taps.tap[t] = (*taps_full)[t];
+        if (t < kMaxTaps) {
+            p->taps.tap[t] = (*taps_full)[t];
+            p->taps64.tap[t] = make_double2((double)v.real(), (double)v.imag());
+        }
     }
     memset(&p->phase, 0, sizeof(p->phase));
     twiddle->resize(kMaxN);
@@ -89,6 +94,7 @@ int build_cyclic_tables(draco_plan* p, std::vector<float2>* taps_full, std::vect
     for (int j = 0; j < n; ++j) {
         const cld ph = root_of_unity(n, (long long)j * M);
         p->phase.phase[j] = make_float2((float)ph.real(), (float)ph.imag());
+        p->phase64.phase[j] = make_double2((double)ph.real(), (double)ph.imag());
         const cld tw = root_of_unity(n, j);
         (*twiddle)[j] = make_double2((double)tw.real(), (double)tw.imag());
     }
@@ -125,7 +131,7 @@ int draco_plan_create(int n, int s, int64_t d, int code, draco_plan** out) {
     draco_plan* p = new (std::nothrow) draco_plan();
     if (!p) return DRACO_ENOMEM;
     memset(p, 0, sizeof(*p));
-    p->n = n; p->s = s; p->d = d; p->code = code; p->theta = 1e-4;
+    p->n = n; p->s = s; p->d = d; p->code = code; p->theta = 1e-6;
     cudaError_t err = cudaGetDevice(&p->device);
     if (err == cudaSuccess) err = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
     if (err != cudaSuccess) { free_plan(p); return cuda_fail(err, "cudaGetDevice"); }
@@ -278,7 +284,9 @@ int draco_get_info(draco_plan* plan, draco_info* info, void* stream) {
     info->no_majority = h.no_majority;
     info->scale = h.scale;
     info->max_syndrome = h.max_syndrome;
-    return DRACO_OK;
+    info->internal_error = h.internal_error;
+    info->reserved = 0;
+    return h.internal_error ? DRACO_EINTERNAL : DRACO_OK;
 }
 
 int draco_generate(float* out, int rows, int64_t len, int row0, float mean, float std, uint64_t seed, void* stream) {
@@ -372,6 +380,7 @@ const char* draco_strerror(int code) {
         case DRACO_ECUDA: return "CUDA runtime error";
         case DRACO_ETOOMANY: return "more than 2 s nodes flagged: no decode vector exists";
         case DRACO_ENOMEM: return "out of memory";
+        case DRACO_EINTERNAL: return "a bounded wait inside a kernel expired";
         case DRACO_ENOMAJ: return "no strict majority at some coordinate";
         default: return "unknown code";
     }

@@ -28,6 +28,14 @@ struct EncodePhase {
     float2 phase[kMaxN];
 };
 
+struct EncodeTaps64 {                 // the same taps / phases in fp64 (centre taps and the final rotation)
+    double2 tap[kMaxTaps];
+};
+
+struct EncodePhase64 {
+    double2 phase[kMaxN];
+};
+
 // Device-resident state of the cyclic decoder (lives in the plan's scratch).
 struct CycDevice {
     double2 twiddle[kMaxN];           // w^k, w = exp(2 pi i / n)
@@ -50,6 +58,8 @@ struct DeviceInfo {                   // mirrors draco_info
     unsigned long long no_majority;
     double scale;
     double max_syndrome;
+    int32_t internal_error;
+    int32_t reserved;
 };
 
 }  // namespace draco
@@ -66,6 +76,8 @@ struct draco_plan {
     double* W_host;                   // [n][n][2]
     draco::EncodeTaps taps;
     draco::EncodePhase phase;
+    draco::EncodeTaps64 taps64;
+    draco::EncodePhase64 phase64;
     float2* taps_full_dev;            // generic encoder: taps for any s, device [2s+1]
     // device scratch
     draco::CycDevice* cyc_dev;
