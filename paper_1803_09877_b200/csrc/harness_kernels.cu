@@ -44,21 +44,33 @@ generate_kernel(float* __restrict__ out, int rows, int64_t len, int64_t ld, int6
     }
 }
 
+__device__ __forceinline__ float corrupt_value(float v, int64_t idx, int model, float param, uint64_t key, int is_complex,
+                                               float inv_sigma) {
+    if (model == DRACO_ADV_REVGRAD) return __fmul_rn(v, -param);
+    if (model == DRACO_ADV_CONST) return (is_complex && (idx & 1)) ? 0.0f : param;
+    return __fadd_rn(v, __fmul_rn(approx_normal(key, (uint64_t)idx, inv_sigma), param));
+}
+
+// One adversarial row, in place; VEC = 4 when the row slice is 16-byte aligned and a multiple of 4 values.
+template <int VEC>
 __global__ void __launch_bounds__(kThreads)
 corrupt_kernel(float* __restrict__ row, int64_t nvals, int64_t v0, int model, float param, uint64_t key, int is_complex,
                float inv_sigma) {
     const int64_t stride = (int64_t)gridDim.x * kThreads;
-    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < nvals; i += stride) {
-        float v;
-        if (model == DRACO_ADV_REVGRAD) {
-            v = __fmul_rn(row[i], -param);
-        } else if (model == DRACO_ADV_CONST) {
-            v = (is_complex && ((v0 + i) & 1)) ? 0.0f : param;
-        } else {
-            const float x = approx_normal(key, (uint64_t)(v0 + i), inv_sigma);
-            v = __fadd_rn(row[i], __fmul_rn(x, param));
+    if (VEC == 4) {
+        float4* row4 = reinterpret_cast<float4*>(row);
+        for (int64_t q = (int64_t)blockIdx.x * kThreads + threadIdx.x; q < nvals / 4; q += stride) {
+            float4 v = model == DRACO_ADV_CONST ? make_float4(0.f, 0.f, 0.f, 0.f) : __ldcs(row4 + q);
+            const int64_t i = v0 + q * 4;
+            v.x = corrupt_value(v.x, i, model, param, key, is_complex, inv_sigma);
+            v.y = corrupt_value(v.y, i + 1, model, param, key, is_complex, inv_sigma);
+            v.z = corrupt_value(v.z, i + 2, model, param, key, is_complex, inv_sigma);
+            v.w = corrupt_value(v.w, i + 3, model, param, key, is_complex, inv_sigma);
+            __stcs(row4 + q, v);
         }
-        row[i] = v;
+    } else {
+        for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < nvals; i += stride)
+            row[i] = corrupt_value(row[i], v0 + i, model, param, key, is_complex, inv_sigma);
     }
 }
 
@@ -90,8 +102,13 @@ int launch_generate(float* out, int rows, int64_t len, int64_t ld, int64_t i0, i
 int launch_corrupt_row(float* row, int64_t nvals, int64_t v0, int model, float param, uint64_t seed, int node,
                        bool is_complex, cudaStream_t st) {
     const uint64_t key = host_splitmix64_at(seed, (uint64_t)node);
-    corrupt_kernel<<<grid_for(nvals), kThreads, 0, st>>>(row, nvals, v0, model, param, key, is_complex ? 1 : 0,
-                                                         inv_sigma_f32());
+    const bool vec4 = (nvals % 4 == 0) && ((reinterpret_cast<uintptr_t>(row) & 15u) == 0);
+    if (vec4)
+        corrupt_kernel<4><<<grid_for(nvals / 4), kThreads, 0, st>>>(row, nvals, v0, model, param, key, is_complex ? 1 : 0,
+                                                                    inv_sigma_f32());
+    else
+        corrupt_kernel<1><<<grid_for(nvals), kThreads, 0, st>>>(row, nvals, v0, model, param, key, is_complex ? 1 : 0,
+                                                                inv_sigma_f32());
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }
