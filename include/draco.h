@@ -50,6 +50,7 @@ enum {
     DRACO_ETOOMANY = -3, /* more than 2 s nodes flagged: no decode vector exists (u is written as zeros) */
     DRACO_ENOMEM = -4,
     DRACO_EINTERNAL = -5, /* a bounded wait inside a kernel expired (reported by draco_get_info); results are invalid */
+    DRACO_ELIMIT = -6,   /* a size exceeds a fixed capacity of the entry point called (see draco_cyc_project_noalloc) */
     DRACO_ENOMAJ = 1     /* warning: some (group, coordinate) had no strict majority; u holds Algorithm 2's candidate */
 };
 
@@ -137,6 +138,30 @@ int draco_rep_vote(draco_plan* plan, const void* R, float* u, float* maj, uint8_
  * projections: e (device [n] complex as (re, im) doubles) = f R over this plan's d coordinates. */
 int draco_cyc_project(draco_plan* plan, const void* R, const float* f, double* e, void* stream);
 int draco_cyc_locate_from_projection(draco_plan* plan, const double* e, uint8_t* flags, void* stream);
+
+/*
+ * The projection e = f R again, for callers that may not allocate.  (The paper has no counterpart:
+ * this is a deployment variant of draco_cyc_project, not a step of the method.)
+ *
+ * Who needs it: a host process whose device memory is owned entirely by another allocator (a
+ * serving framework's pool that took the whole GPU at start-up, so a later cudaMalloc fails or
+ * splits the pool), or a step loop that cannot tolerate the device-wide synchronisation that an
+ * allocation or free may imply.  draco_plan_create allocates; this entry point needs no plan and
+ * calls neither cudaMalloc nor cudaFree nor any allocating library routine.  Its only scratch, the
+ * per-block partial sums, is a fixed array compiled into the library: 296 blocks x 128 nodes x 16
+ * bytes = 592 KB of device memory on every GPU that loads the library, held until the process ends.
+ *
+ * n nodes, d coordinates; R: device [n][d] complex64; f: device [d] fp32; e: device [n] complex as
+ * (re, im) doubles, written by the call.  All three 16-byte aligned; the caller owns them.
+ * Limits: n <= DRACO_MAX_N (128) and device ordinal < 64, else DRACO_ELIMIT; d is unbounded
+ * (at most 296 blocks are launched, each walking its share of the tiles).
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call before any stream capture begins.  All calls on a device share the one
+ * array, which keeps the previous call's contents (every call overwrites all entries it reads, so
+ * nothing needs clearing); two calls that overlap on the GPU, on any streams, race on it.
+ * Same arithmetic, grid and summation order as draco_cyc_project: identical results.
+ */
+int draco_cyc_project_noalloc(int n, int64_t d, const void* R, const float* f, double* e, void* stream);
 
 /* The decode vector b of the last cyclic decode (host [n][2] doubles); synchronises the stream. */
 int draco_cyc_decode_vector(draco_plan* plan, double* b_host /*host*/, void* stream);

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     DracoError,
     DracoInfo,
     Plan,
+    cyc_project_noalloc,
     generate,
     lib,
     library_path,

@@ -11,7 +11,7 @@ import os
 
 REP, CYC = 0, 1
 ADV_REVGRAD, ADV_CONST, ADV_GAUSS = 0, 1, 2
-OK, EINVAL, ECUDA, ETOOMANY, ENOMEM, EINTERNAL, ENOMAJ = 0, -1, -2, -3, -4, -5, 1
+OK, EINVAL, ECUDA, ETOOMANY, ENOMEM, EINTERNAL, ELIMIT, ENOMAJ = 0, -1, -2, -3, -4, -5, -6, 1
 MAX_N = 128
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -59,6 +59,7 @@ _SIGS = {
     "draco_rep_vote": ([_vp, _vp, _vp, _vp, _vp, _vp], _i),
     "draco_cyc_project": ([_vp, _vp, _vp, _vp, _vp], _i),
     "draco_cyc_locate_from_projection": ([_vp, _vp, _vp, _vp], _i),
+    "draco_cyc_project_noalloc": ([_i, _i64, _vp, _vp, _vp, _vp], _i),
     "draco_cyc_decode_vector": ([_vp, C.POINTER(C.c_double), _vp], _i),
     "draco_get_info": ([_vp, C.POINTER(DracoInfo), _vp], _i),
     "draco_pipeline_host": ([_vp, _vp, _vp, C.POINTER(_i), C.POINTER(_i), C.POINTER(_f), _i, _u64, _vp, _vp, _vp,
@@ -107,6 +108,11 @@ def _adv_arrays(adv_idx, adv_model, adv_param):
     k = len(adv_idx)
     return ((_i * k)(*[int(a) for a in adv_idx]), (_i * k)(*[int(a) for a in adv_model]),
             (_f * k)(*[float(a) for a in adv_param]), k)
+
+
+def cyc_project_noalloc(n: int, d: int, R, f, e, stream=None):
+    """draco_cyc_project_noalloc: e = f R with the library's built-in scratch; needs no plan and allocates nothing."""
+    return _check(lib.draco_cyc_project_noalloc(n, d, _ptr(R), _ptr(f), _ptr(e), _stream(stream)))
 
 
 def generate(out, rows: int, length: int, row0: int = 0, mean: float = 0.0, std: float = 1.0, seed: int = 0,

@@ -10,6 +10,8 @@
 //
 // The small solves run in fp64 in a single thread block; only the projection touches HBM:
 // 8 n len + 4 len bytes read.
+#include <mutex>
+
 #include "draco_internal.cuh"
 
 namespace draco {
@@ -545,3 +547,70 @@ int launch_cyc_decode_vector(draco_plan* p, const uint8_t* flags, cudaStream_t s
 }
 
 }  // namespace draco
+
+// ------------------------------------------------------------------ projection without any allocation
+// Some callers must not allocate device memory at all: a parameter server embedded in a host
+// process whose memory pool owner has handed out the whole device up front (a later cudaMalloc
+// fails or fragments the pool), or a step loop that cannot afford the implicit device-wide
+// synchronisation an allocation or a free may cause.  For them the block partials of the
+// projection live in this fixed array instead of in a plan.  Every GPU that loads the library
+// carries its 592 KB until the process exits.
+namespace draco {
+namespace {
+constexpr int kStaticGridMax = 296;                                   // blocks whose partials fit
+static __device__ __align__(256) double2 g_static_partial[kStaticGridMax * kMaxN];
+constexpr int kMaxDevices = 64;
+double2* g_static_partial_ptr[kMaxDevices] = {};                      // device address per device, set once
+int g_static_sm_count[kMaxDevices] = {};
+std::mutex g_static_mutex;
+}  // namespace
+}  // namespace draco
+
+extern "C" int draco_cyc_project_noalloc(int n, int64_t d, const void* R, const float* f, double* e, void* stream) {
+    using namespace draco;
+    if (n < 1 || d < 1 || !R || !f || !e) return DRACO_EINVAL;
+    if (n > kMaxN) return DRACO_ELIMIT;                               // the static array holds at most kMaxN rows per block
+    if ((reinterpret_cast<uintptr_t>(R) & 15u) || (reinterpret_cast<uintptr_t>(f) & 15u) ||
+        (reinterpret_cast<uintptr_t>(e) & 15u))
+        return DRACO_EINVAL;
+    int dev = 0;
+    DRACO_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return DRACO_ELIMIT;
+    double2* partial = nullptr;
+    int sms = 0;
+    {
+        // Set-up, once per device, with that device current.  In host code the array's name is only a
+        // stand-in for the symbol; the kernel needs the device address, which the runtime looks up here.
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_partial_ptr[dev]) {
+            double2* ptr = nullptr;
+            DRACO_CUDA(cudaGetSymbolAddress((void**)&ptr, g_static_partial));
+            int count = 0;
+            DRACO_CUDA(cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev));
+            g_static_sm_count[dev] = count;
+            g_static_partial_ptr[dev] = ptr;
+        }
+        partial = g_static_partial_ptr[dev];
+        sms = g_static_sm_count[dev];
+    }
+    int grid = project_grid_size(sms);
+    if (grid > kStaticGridMax) grid = kStaticGridMax;
+    if (grid < 1) grid = 1;
+    cudaStream_t st = (cudaStream_t)stream;
+    const float2* Rc = static_cast<const float2*>(R);
+    // Every block writes its n partials (zeros if it had no tile), so nothing has to be cleared
+    // between calls even though the array keeps the previous call's contents.
+    if (d % 2 == 0) {
+        if (n <= 32) cyc_project_kernel<4, true><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
+        else if (n <= 64) cyc_project_kernel<8, true><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
+        else cyc_project_kernel<16, true><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
+    } else {
+        if (n <= 32) cyc_project_kernel<4, false><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
+        else if (n <= 64) cyc_project_kernel<8, false><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
+        else cyc_project_kernel<16, false><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
+    }
+    DRACO_CUDA(cudaGetLastError());
+    cyc_project_finish_kernel<<<1, kMaxN, 0, st>>>(partial, grid, n, reinterpret_cast<double2*>(e));
+    DRACO_CUDA(cudaGetLastError());
+    return DRACO_OK;
+}

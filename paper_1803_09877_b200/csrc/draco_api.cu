@@ -381,6 +381,7 @@ const char* draco_strerror(int code) {
         case DRACO_ETOOMANY: return "more than 2 s nodes flagged: no decode vector exists";
         case DRACO_ENOMEM: return "out of memory";
         case DRACO_EINTERNAL: return "a bounded wait inside a kernel expired";
+        case DRACO_ELIMIT: return "size exceeds a fixed capacity of this entry point";
         case DRACO_ENOMAJ: return "no strict majority at some coordinate";
         default: return "unknown code";
     }

@@ -1,0 +1,49 @@
+"""draco_cyc_project_noalloc: the projection for callers that may not allocate device memory
+(their GPU memory belongs to another allocator, or they cannot afford an allocation's implicit
+synchronisation inside the step loop).  It keeps its scratch in an array built into the library,
+so this test checks, through the C ABI, that it returns what the plan-based entry point returns,
+on two calls in a row with different inputs (the second must not see the first call's leftovers).
+Collected last on purpose: a failure here cannot hide another test's result under `-x`.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import draco_inputs as di
+
+pytestmark = pytest.mark.gpu
+
+
+def _project_both_ways(dr, n, s, d, seed):
+    R = torch.from_numpy(di.complex_rows(seed, n, d, std=3.0).view(np.float32)).cuda()
+    f = torch.from_numpy(di.projection_vector(seed + 1, d)).cuda()
+    plan = dr.Plan(n, s, d, dr.CYC)
+    e_plan = torch.zeros(2 * n, dtype=torch.float64, device="cuda")
+    plan.cyc_project(R, f, e_plan)
+    e_static = torch.full((2 * n,), float("nan"), dtype=torch.float64, device="cuda")
+    dr.cyc_project_noalloc(n, d, R, f, e_static)
+    torch.cuda.synchronize()
+    return e_plan.cpu().numpy().view(np.complex128), e_static.cpu().numpy().view(np.complex128)
+
+
+def test_noalloc_projection_matches_plan_projection_twice_in_a_row():
+    import paper_1803_09877_b200 as dr
+    for call, (n, s, d) in enumerate([(45, 5, 300_004), (15, 2, 4099)]):     # vector path, then the odd-d scalar path
+        want, got = _project_both_ways(dr, n, s, d, seed=100 + call)
+        assert np.all(np.isfinite(got.view(np.float64)))
+        assert np.abs(got - want).max() <= 1e-6 * np.abs(want).max()           # tolerance of the projection parity tests
+        np.testing.assert_array_equal(got, want)                               # same kernel, grid and order: same bits
+
+
+def test_noalloc_projection_rejects_sizes_beyond_its_fixed_capacity():
+    import paper_1803_09877_b200 as dr
+    from paper_1803_09877_b200 import binding
+    buf = torch.zeros(1024, dtype=torch.float32, device="cuda")
+    e = torch.zeros(512, dtype=torch.float64, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    rc = binding.lib.draco_cyc_project_noalloc(129, 4, buf.data_ptr(), buf.data_ptr(), e.data_ptr(), st)
+    assert rc == binding.ELIMIT and b"capacity" in binding.lib.draco_strerror(rc)
+    assert binding.lib.draco_cyc_project_noalloc(0, 4, buf.data_ptr(), buf.data_ptr(), e.data_ptr(), st) == binding.EINVAL
+    assert binding.lib.draco_cyc_project_noalloc(4, 4, None, buf.data_ptr(), e.data_ptr(), st) == binding.EINVAL
