@@ -159,7 +159,8 @@ int draco_cyc_locate_from_projection(draco_plan* plan, const double* e, uint8_t*
  * make that first call before any stream capture begins.  All calls on a device share the one
  * array, which keeps the previous call's contents (every call overwrites all entries it reads, so
  * nothing needs clearing); two calls that overlap on the GPU, on any streams, race on it.
- * Same arithmetic, grid and summation order as draco_cyc_project: identical results.
+ * Same kernel and arithmetic as draco_cyc_project; only the number of fp64 block partials may differ
+ * (296 at most here), so the two agree to fp64 rounding (about 1e-15 relative).
  */
 int draco_cyc_project_noalloc(int n, int64_t d, const void* R, const float* f, double* e, void* stream);
 

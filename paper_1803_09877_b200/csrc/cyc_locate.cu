@@ -504,7 +504,7 @@ cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n
 
 }  // namespace
 
-int project_grid_size(int sm_count) { return sm_count * 2; }
+int project_grid_size(int sm_count) { return sm_count * 4; }
 
 int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t len, int64_t ld, bool accumulate,
                        cudaStream_t st) {

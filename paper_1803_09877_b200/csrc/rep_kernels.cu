@@ -129,24 +129,51 @@ rep_vote_kernel(const uint32_t* __restrict__ R, int64_t len, int64_t ld, GroupTa
 #pragma unroll
                     for (int c = 0; c < VEC; ++c) sel[c] = val[0].get(c);
                 } else {
+                    // Some replica differs.  A value held by strictly more than half of the group IS
+                    // what Algorithm 2 returns, so first count the votes for member 0's value, then for
+                    // member 1's (member 0 may be the adversary); only if neither has a strict majority
+                    // on all VEC coordinates is the streaming vote itself run.
                     uint32_t dis = 0;
+                    bool settled = false;
 #pragma unroll
-                    for (int c = 0; c < VEC; ++c) {
-                        uint32_t ma = val[0].get(c);
-                        int counter = 0;
+                    for (int ref = 0; ref < 2 && ref < MMAX; ++ref) {
+                        if (!settled && ref < m) {
+                            uint32_t d_ref = 0;
+                            bool all_major = true;
 #pragma unroll
-                        for (int k = 0; k < MMAX; ++k)
-                            if (k < m) vote_step(val[k].get(c), ma, counter);
-                        int votes = 0;
+                            for (int c = 0; c < VEC; ++c) {
+                                const uint32_t cand = val[ref].get(c);
+                                uint32_t ne = 0;
 #pragma unroll
-                        for (int k = 0; k < MMAX; ++k)
-                            if (k < m) {
-                                const bool same = val[k].get(c) == ma;
-                                votes += same;
-                                dis |= (same ? 0u : 1u) << k;
+                                for (int k = 0; k < MMAX; ++k)
+                                    if (k < m) ne |= (val[k].get(c) != cand ? 1u : 0u) << k;
+                                all_major &= (2 * (m - __popc(ne)) > m);
+                                d_ref |= ne;
                             }
-                        nomaj += (2 * votes <= m);
-                        sel[c] = ma;
+                            if (all_major) {
+#pragma unroll
+                                for (int c = 0; c < VEC; ++c) sel[c] = val[ref].get(c);
+                                dis = d_ref;
+                                settled = true;
+                            }
+                        }
+                    }
+                    if (!settled) {
+#pragma unroll
+                        for (int c = 0; c < VEC; ++c) {
+                            uint32_t ma = val[0].get(c);
+                            int counter = 0;
+#pragma unroll
+                            for (int k = 0; k < MMAX; ++k)
+                                if (k < m) vote_step(val[k].get(c), ma, counter);
+                            uint32_t ne = 0;
+#pragma unroll
+                            for (int k = 0; k < MMAX; ++k)
+                                if (k < m) ne |= (val[k].get(c) != ma ? 1u : 0u) << k;
+                            nomaj += (2 * (m - __popc(ne)) <= m);
+                            dis |= ne;
+                            sel[c] = ma;
+                        }
                     }
                     if (dis & ~smask[g][0]) atomicOr(&smask[g][0], dis);
                 }

@@ -34,7 +34,7 @@ def test_noalloc_projection_matches_plan_projection_twice_in_a_row():
         want, got = _project_both_ways(dr, n, s, d, seed=100 + call)
         assert np.all(np.isfinite(got.view(np.float64)))
         assert np.abs(got - want).max() <= 1e-6 * np.abs(want).max()           # tolerance of the projection parity tests
-        np.testing.assert_array_equal(got, want)                               # same kernel, grid and order: same bits
+        assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()          # same kernel; only the number of block partials differs
 
 
 def test_noalloc_projection_rejects_sizes_beyond_its_fixed_capacity():
