@@ -350,6 +350,115 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+
+# --------------------------------------------------------------------------- sweep over both codes
+def run_sweep(args):
+    """Both codes over n x s x d: per point the stage times, GB/s of coded gradients consumed / produced,
+    achieved HBM GB/s against the roofline, and correctness for 0, s and more than s adversaries
+    (the last must fail visibly).  One JSON line per point goes to --sweep-out; one summary line to stdout."""
+    import torch
+
+    import paper_1803_09877_b200 as dr
+
+    torch.cuda.set_device(0)
+    peak, peak_src = measured_peak_gbs()
+    free_bytes = torch.cuda.mem_get_info()[0]
+    ns = [int(x) for x in args.sweep_n.split(",")]
+    ss = [int(x) for x in args.sweep_s.split(",")]
+    ds = [int(float(x)) for x in args.sweep_d.split(",")]
+    rng = np.random.default_rng(7)
+    out_lines, skipped = [], []
+
+    def timed(fn, reps=3):
+        fn()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        for i in range(reps):
+            ev[i].record()
+            fn()
+        ev[reps].record()
+        torch.cuda.synchronize()
+        return statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(reps))
+
+    for code in ("rep", "cyc"):
+        cyc = code == "cyc"
+        for n in ns:
+            for s in ss:
+                if 2 * s + 1 > n:
+                    continue
+                for d in ds:
+                    need = 4 * n * d * (3 if cyc else 2) + 16 * d
+                    if need > 0.92 * free_bytes:
+                        skipped.append({"code": code, "n": n, "s": s, "d": d, "reason": f"needs {need / 1e9:.0f} GB"})
+                        continue
+                    seed = SEED + 100 * n + s
+                    plan = dr.Plan(n, s, d, dr.CYC if cyc else dr.REP)
+                    G = torch.empty((n, d), dtype=torch.float32, device="cuda")
+                    dr.generate(G, n, d, seed=seed)
+                    f = torch.empty(d, dtype=torch.float32, device="cuda")
+                    dr.generate(f, 1, d, mean=1.0, std=1.0, seed=seed + 3)
+                    Z = torch.empty((n, (2 if cyc else 1) * d), dtype=torch.float32, device="cuda")
+                    u = torch.empty(d, dtype=torch.float32, device="cuda")
+                    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+                    idx = np.unique(rng.integers(0, d, 2000))
+                    exact = di.gradient_rows(seed, n, d, idx=idx).astype(np.float64).sum(axis=0)
+                    scale = max(float(np.abs(exact).max()), 1e-30)
+                    groups = plan.groups() if not cyc else []
+                    checks = {}
+                    for label in ("0", "s", ">s"):
+                        if label == "0":
+                            adv, model, param = [], [], []
+                        elif label == "s":
+                            adv = di.choose_adversaries(seed + 1, n, s).tolist()
+                            model, param = [di.ADV_REVGRAD] * s, [100.0] * s
+                        elif cyc:
+                            adv = di.choose_adversaries(seed + 2, n, s + 1).tolist()
+                            model, param = [di.ADV_REVGRAD] * (s + 1), [100.0] * (s + 1)
+                        else:                      # enough identical colluders to win group 0's vote
+                            c = groups[0][1] // 2 + 1
+                            adv, model, param = list(range(c)), [di.ADV_CONST] * c, [1e4] * c
+                        plan.encode(G, Z)
+                        if adv:
+                            plan.corrupt(Z, adv, model, param, seed=seed + 4)
+                        plan.locate_decode(Z, f if cyc else None, flags, u)
+                        info = plan.info()
+                        got = sorted(np.flatnonzero(flags.cpu().numpy()).tolist())
+                        err = float(np.abs(u[idx].cpu().numpy().astype(np.float64) - exact).max() / scale)
+                        checks[label] = {"planted": len(adv), "flags_match": got == sorted(adv), "err": err,
+                                         "status": info["status"], "no_majority": info["no_majority"]}
+                    adv = di.choose_adversaries(seed + 1, n, s).tolist()
+                    enc_ms = timed(lambda: plan.encode(G, Z))
+                    if adv:
+                        plan.corrupt(Z, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 4)
+                    dec_ms = timed(lambda: plan.locate_decode(Z, f if cyc else None, flags, u))
+                    ab = algorithmic_bytes(code, n, s, d, len(adv))
+                    enc_hbm = ab["encode"] / (enc_ms * 1e-3) / 1e9
+                    dec_hbm = (ab["locate"] + ab["decode"]) / (dec_ms * 1e-3) / 1e9
+                    tol = 1e-5 if not cyc else (1e-4 if n <= 15 else None)
+                    ok_s = checks["s"]["flags_match"] and checks["0"]["flags_match"]
+                    line = {"code": code, "n": n, "s": s, "d": d, "encode_ms": enc_ms, "decode_ms": dec_ms,
+                            "coded_GBps_produced": ab["coded"] / (enc_ms * 1e-3) / 1e9,
+                            "coded_GBps_consumed": ab["coded"] / (dec_ms * 1e-3) / 1e9,
+                            "encode_hbm_GBps": enc_hbm, "encode_frac": enc_hbm / peak,
+                            "decode_hbm_GBps": dec_hbm, "decode_frac": dec_hbm / peak,
+                            "l2_note": "fits in L2: not an HBM number" if ab["coded"] < 2.5e8 else "",
+                            "checks": checks, "flags_ok_upto_s": ok_s, "sum_tolerance": tol,
+                            "sum_ok_upto_s": None if tol is None else (checks["0"]["err"] <= tol and checks["s"]["err"] <= tol),
+                            "beyond_s_fails": (not checks[">s"]["flags_match"]) or checks[">s"]["err"] > 1e-3
+                            or checks[">s"]["status"] != 0}
+                    out_lines.append(line)
+                    with open(args.sweep_out, "a") as fh:
+                        fh.write(json.dumps(line) + "\n")
+                    del G, Z, u, f, plan
+                    torch.cuda.empty_cache()
+    big = [x for x in out_lines if not x["l2_note"] and x["d"] >= 11_000_000]
+    summary = {"mode": "sweep", "points": len(out_lines), "skipped": skipped, "peak_GBps": peak, "peak_source": peak_src,
+               "flags_ok_upto_s": sum(bool(x["flags_ok_upto_s"]) for x in out_lines),
+               "beyond_s_fails": sum(bool(x["beyond_s_fails"]) for x in out_lines),
+               "min_decode_frac_large_d": min((x["decode_frac"] for x in big), default=None),
+               "min_encode_frac_large_d": min((x["encode_frac"] for x in big), default=None), "out": args.sweep_out}
+    print(json.dumps(summary))
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -358,6 +467,11 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--d", type=int, default=None, help="override the workload's d (profiling on a small case)")
+    ap.add_argument("--sweep", action="store_true", help="both codes over n x s x d (one GPU); JSON lines to --sweep-out")
+    ap.add_argument("--sweep-n", default="15,45,105")
+    ap.add_argument("--sweep-s", default="1,2,5,7")
+    ap.add_argument("--sweep-d", default="1e6,11.7e6,60.2e6,138e6")
+    ap.add_argument("--sweep-out", default=os.path.join(ROOT, "gpurun_out", "sweep.jsonl"))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -366,7 +480,10 @@ def main():
         w[3] = args.d
         args.workload = f"{args.workload}@d={args.d}"
         WORKLOADS[args.workload] = tuple(w)
-    if args.impl == "reference":
+    if args.sweep:
+        os.makedirs(os.path.dirname(args.sweep_out), exist_ok=True)
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

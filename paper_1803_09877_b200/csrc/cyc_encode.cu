@@ -11,10 +11,10 @@
 // rotation per output.  The taps do not depend on j, so they sit in the kernel's constant
 // parameter bank and every multiply-add takes its coefficient from there.
 //
-// Data movement.  A thread block owns a tile of 1024 coordinates and walks the n rows once.
-// One producer lane streams the row tiles (4 KB each) from global memory into a ring of
+// Data movement.  A thread block owns a tile of 1536 coordinates and walks the n rows once.
+// One producer lane streams the row tiles (6 KB each) from global memory into a ring of
 // shared-memory stages with bulk asynchronous copies (cp.async.bulk + mbarrier, no
-// multicast); 8 consumer warps take each row from the ring into a register window of the
+// multicast); 12 consumer warps take each row from the ring into a register window of the
 // last 2 s + 1 rows, 4 coordinates per thread.  The first 2 s rows are also kept in shared
 // memory, because the circle closes on them at the end of the walk; nothing is read twice.
 // HBM traffic is the algorithmic minimum: 4 n len bytes read + 8 n len bytes written.
@@ -31,11 +31,12 @@ namespace draco {
 
 namespace {
 
-constexpr int kConsumers = 256;                 // consumer threads (8 warps); warp 8 is the producer
+constexpr int kConsumers = 384;                 // consumer threads (12 warps); the next warp is the producer
 constexpr int kRingThreads = kConsumers + 32;
 constexpr int kVec = 4;                         // coordinates per consumer thread
 constexpr int kTile = kConsumers * kVec;        // coordinates per tile = floats per stage
-constexpr int kStages = 16;                     // ring depth (64 KB in flight per block)
+constexpr int kStages = 16;                     // ring depth (96 KB in flight per block)
+static_assert((kStages & (kStages - 1)) == 0, "stage indices and parities are derived with masks: kStages must be a power of two");
 constexpr int kGenericThreads = 256;
 
 // ---------------------------------------------------------------- mbarrier / bulk-copy wrappers
