@@ -104,7 +104,8 @@ def oracle_threads():
 
 def cpu_baseline(workload, target_seconds=15.0):
     code, n, s, d, std, models, params = WORKLOADS[workload]
-    probe = min(d, 100_000)
+    probe = min(d, 200_000)
+    oracle_step(workload, probe, SEED)                                   # builds and caches the code tables
     dt, _ = oracle_step(workload, probe, SEED)
     d_sample = int(min(d, max(probe, probe * target_seconds / max(dt, 1e-3))))
     dt, ok = oracle_step(workload, d_sample, SEED)
@@ -121,6 +122,7 @@ def run_reference(args):
     workload = args.workload
     code, n, s, d, std, models, params = WORKLOADS[workload]
     probe = min(d, 50_000)
+    oracle_step(workload, probe, SEED)                                   # builds and caches the code tables
     dt, _ = oracle_step(workload, probe, SEED)
     budget = 150.0 / max(1, args.steps + args.warmup)                  # seconds per step
     d_sample = int(min(d, max(10_000, probe * min(budget, 3.0) / max(dt, 1e-3))))
@@ -380,7 +382,7 @@ def run_sweep(args):
         torch.cuda.synchronize()
         return statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(reps))
 
-    for code in ("rep", "cyc"):
+    for code in args.sweep_codes.split(","):
         cyc = code == "cyc"
         for n in ns:
             for s in ss:
@@ -468,6 +470,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--d", type=int, default=None, help="override the workload's d (profiling on a small case)")
     ap.add_argument("--sweep", action="store_true", help="both codes over n x s x d (one GPU); JSON lines to --sweep-out")
+    ap.add_argument("--sweep-codes", default="rep,cyc")
     ap.add_argument("--sweep-n", default="15,45,105")
     ap.add_argument("--sweep-s", default="1,2,5,7")
     ap.add_argument("--sweep-d", default="1e6,11.7e6,60.2e6,138e6")

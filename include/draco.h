@@ -11,7 +11,9 @@
  * Layout.  Every matrix is worker-major and dense: row k of G is gradient g_k
  * (d contiguous fp32), row j of Z / R is node j's vector: d fp32 for the
  * repetition code, d interleaved (re, im) fp32 pairs (complex64) for the cyclic
- * code.  u is d fp32.  Indices are 0-based.  Row stride = d elements.
+ * code (DRACO_CYC_PACKED: ceil(d / 2) such pairs, entry i holding gradient coordinates i and
+ * ceil(d / 2) + i; the decoder returns [Re(u-hat); Im(u-hat)] cut to d entries).  u is d fp32.
+ * Indices are 0-based.  Row stride = the row length.
  *
  * Ownership.  The caller owns every buffer it passes (device buffers unless a
  * parameter says "host"); the library never frees or keeps them.  A plan owns
@@ -39,7 +41,12 @@ extern "C" {
 typedef struct draco_plan draco_plan;
 
 /* code type */
-enum { DRACO_REP = 0, DRACO_CYC = 1 };
+enum {
+    DRACO_REP = 0,        /* repetition code, fp32 vectors of d entries */
+    DRACO_CYC = 1,        /* cyclic code, complex64 vectors of d entries */
+    DRACO_CYC_PACKED = 2  /* cyclic code on the packed gradient (Section 3, last paragraph): complex64 vectors of
+                             ceil(d / 2) entries, entry i = (G_i, G_{ceil(d/2)+i}); f has ceil(d / 2) entries; u has d */
+};
 /* adversary models of the corruptor (Section 4, "Adversarial Attack Models", plus Gaussian noise) */
 enum { DRACO_ADV_REVGRAD = 0, DRACO_ADV_CONST = 1, DRACO_ADV_GAUSS = 2 };
 /* return codes */

@@ -364,3 +364,46 @@ def cyc_decode_full(R: np.ndarray, f: np.ndarray, n: int, s: int, theta: float =
     loc = cyc_locate(R, f, n, s, theta)
     loc["u"] = cyc_decode(R, n, s, loc["flags"]) if loc["flags"].sum() <= 2 * s else None
     return loc
+
+
+# --------------------------------------------------------------------------
+# Real -> complex packing of the cyclic code  (Section 3, last paragraph)
+# --------------------------------------------------------------------------
+
+
+def cyc_pack(G: np.ndarray) -> np.ndarray:
+    """G-hat in C^{ceil(d/2) x P}: component i has real part G_i and imaginary part
+    G_{ceil(d/2)+i} (zero where d is odd and the second half is one short).
+    Worker-major like everything else: returns ``[n][ceil(d/2)]`` complex128."""
+    G = np.asarray(G, dtype=np.float64)
+    n, d = G.shape
+    h = (d + 1) // 2
+    out = np.zeros((n, h), dtype=np.complex128)
+    out.real = G[:, :h]
+    out.imag[:, : d - h] = G[:, h:]
+    return out
+
+
+def cyc_unpack(u_hat: np.ndarray, d: int) -> np.ndarray:
+    """Inverse of the packing applied to the recovered u-hat = G-hat 1_P.
+
+    The paper writes u = Re(u-hat) + Im(u-hat), which cannot undo a packing that put
+    different coordinates in the two parts; the reading taken is the concatenation
+    [Re(u-hat); Im(u-hat)] cut to d entries."""
+    h = (d + 1) // 2
+    u_hat = np.asarray(u_hat, dtype=np.complex128)
+    return np.concatenate([u_hat.real, u_hat.imag[: d - h]])
+
+
+def cyc_encode_packed(G: np.ndarray, n: int, s: int, W: np.ndarray | None = None,
+                      dtype=np.complex64) -> np.ndarray:
+    """The compute nodes send G-hat W: ``[n][ceil(d/2)]`` complex."""
+    if W is None:
+        W = cyc_W(n, s)
+    return (W.T @ cyc_pack(G)).astype(dtype)
+
+
+def cyc_decode_packed(R: np.ndarray, n: int, s: int, flags, d: int) -> np.ndarray:
+    """Algorithm 1 steps 2-4 on packed vectors: u-hat = R_{., U} b, then unpack."""
+    b = cyc_decode_vector(n, s, flags)
+    return cyc_unpack(cyc_recover(R, b), d)

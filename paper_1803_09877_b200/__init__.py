@@ -8,7 +8,7 @@ There is no CPU fallback: the first use of any name below loads ``libdraco.so``
 and raises if it has not been built (``python -m paper_1803_09877_b200.build``).
 The ``build`` submodule itself imports without the library.
 """
-_BINDING_NAMES = ("ADV_CONST", "ADV_GAUSS", "ADV_REVGRAD", "CYC", "REP", "DracoError", "DracoInfo", "Plan",
+_BINDING_NAMES = ("ADV_CONST", "ADV_GAUSS", "ADV_REVGRAD", "CYC", "CYC_PACKED", "REP", "DracoError", "DracoInfo", "Plan",
                   "cyc_project_noalloc", "generate", "lib", "library_path")
 __all__ = list(_BINDING_NAMES) + ["binding", "build", "sharding"]
 

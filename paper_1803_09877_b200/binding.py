@@ -9,7 +9,7 @@ from __future__ import annotations
 import ctypes as C
 import os
 
-REP, CYC = 0, 1
+REP, CYC, CYC_PACKED = 0, 1, 2
 ADV_REVGRAD, ADV_CONST, ADV_GAUSS = 0, 1, 2
 OK, EINVAL, ECUDA, ETOOMANY, ENOMEM, EINTERNAL, ELIMIT, ENOMAJ = 0, -1, -2, -3, -4, -5, -6, 1
 MAX_N = 128

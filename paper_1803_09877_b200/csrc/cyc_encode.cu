@@ -106,7 +106,7 @@ struct RingState {
 // MODE 0: first SL steps of a tile (all rows from the ring; outputs from step 2 S on; nothing
 //         pending at step 0);  MODE 1: steady state (ring row + output, previous stage pending);
 // MODE 2: anything (run-time guards).  Returns false when a wait gave up.
-template <int S, int P, int MODE>
+template <int S, int P, int MODE, bool PACKED>
 __device__ __forceinline__ bool encode_step(Window<S>& w, RingState& rs, int vv, int n, const float* ring_t,
                                             float* stash_t, float2* zcol, int64_t ldz, bool active, int lane,
                                             const EncodeTaps& taps, const EncodeTaps64& taps64,
@@ -125,7 +125,13 @@ __device__ __forceinline__ bool encode_step(Window<S>& w, RingState& rs, int vv,
     if (from_ring) {
         const uint32_t bar = rs.full0 + 8 * rs.st;
         if (!mbar_wait(bar, rs.par)) return false;
-        x = *reinterpret_cast<const float4*>(ring_t + rs.st * kTile);
+        if (PACKED) {      // first half of the gradient -> real parts, second half -> imaginary parts
+            const float2 a = *reinterpret_cast<const float2*>(ring_t + rs.st * kTile);
+            const float2 b = *reinterpret_cast<const float2*>(ring_t + rs.st * kTile + kTile / 2);
+            x = make_float4(a.x, a.y, b.x, b.y);
+        } else {
+            x = *reinterpret_cast<const float4*>(ring_t + rs.st * kTile);
+        }
         rs.pend_bar = rs.empty0 + 8 * rs.st;
         rs.pend_bits = __float_as_uint(x.x);
         rs.pending = true;
@@ -175,38 +181,49 @@ __device__ __forceinline__ bool encode_step(Window<S>& w, RingState& rs, int vv,
             for (int c = 0; c < 4; ++c) { dr[c] = fma(cr, w.cw[q][c], dr[c]); di[c] = fma(ci, w.cw[q][c], di[c]); }
         }
         const double2 rot = ph64.phase[j];
-        float zr[4], zi[4];
+        double xr[4], xi[4];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            zr[c] = (float)fma(dr[c], rot.x, -di[c] * rot.y);
-            zi[c] = (float)fma(dr[c], rot.y, di[c] * rot.x);
+            xr[c] = fma(dr[c], rot.x, -di[c] * rot.y);
+            xi[c] = fma(dr[c], rot.y, di[c] * rot.x);
         }
-        if (active) {
+        if (PACKED) {
+            // components 0,1 filtered the real parts (X), 2,3 the imaginary parts (Y): z = X + i Y
+            if (active) {
+                float4* dst = reinterpret_cast<float4*>(zcol + (int64_t)j * ldz);
+                __stcs(dst, make_float4((float)(xr[0] - xi[2]), (float)(xi[0] + xr[2]), (float)(xr[1] - xi[3]),
+                                        (float)(xi[1] + xr[3])));
+            }
+        } else if (active) {
             float4* dst = reinterpret_cast<float4*>(zcol + (int64_t)j * ldz);
-            __stcs(dst, make_float4(zr[0], zi[0], zr[1], zi[1]));
-            __stcs(dst + 1, make_float4(zr[2], zi[2], zr[3], zi[3]));
+            __stcs(dst, make_float4((float)xr[0], (float)xi[0], (float)xr[1], (float)xi[1]));
+            __stcs(dst + 1, make_float4((float)xr[2], (float)xi[2], (float)xr[3], (float)xi[3]));
         }
     }
     return true;
 }
 
-template <int S, int MODE, int P = 0>
+template <int S, int MODE, bool PACKED, int P = 0>
 __device__ __forceinline__ bool encode_chunk(Window<S>& w, RingState& rs, int v0, int n, const float* ring_t,
                                              float* stash_t, float2* zcol, int64_t ldz, bool active, int lane,
                                              const EncodeTaps& taps, const EncodeTaps64& taps64,
                                              const EncodePhase64& ph64) {
     if constexpr (P < Window<S>::SL) {
-        if (!encode_step<S, P, MODE>(w, rs, v0 + P, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64))
+        if (!encode_step<S, P, MODE, PACKED>(w, rs, v0 + P, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64))
             return false;
-        return encode_chunk<S, MODE, P + 1>(w, rs, v0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
+        return encode_chunk<S, MODE, PACKED, P + 1>(w, rs, v0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
     } else {
         return true;
     }
 }
 
-template <int S>
+// PACKED: the real -> complex packing of Section 3's last paragraph.  `len` then counts complex
+// coordinates, a tile holds kTile / 2 of them, and a stage receives two slices of each row:
+// G[r][c0 ..] (real parts) and G[r][half + c0 ..] (imaginary parts).
+template <int S, bool PACKED>
 __global__ void __launch_bounds__(kRingThreads)
-cyc_encode_ring_kernel(const float* __restrict__ G, float2* __restrict__ Z, int64_t len, int64_t ldg, int64_t ldz, int n,
+cyc_encode_ring_kernel(const float* __restrict__ G, float2* __restrict__ Z, int64_t len, int64_t ldg, int64_t ldz,
+                       int64_t half, int n,
                        const __grid_constant__ EncodeTaps taps, const __grid_constant__ EncodeTaps64 taps64,
                        const __grid_constant__ EncodePhase64 ph64, int* err) {
     constexpr int SL = Window<S>::SL;
@@ -225,7 +242,9 @@ cyc_encode_ring_kernel(const float* __restrict__ G, float2* __restrict__ Z, int6
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    const int64_t ntiles = (len + kTile - 1) / kTile;
+    constexpr int kTileCoords = PACKED ? kTile / 2 : kTile;      // coordinates of Z per tile
+    constexpr int kPerThread = PACKED ? 2 : kVec;
+    const int64_t ntiles = (len + kTileCoords - 1) / kTileCoords;
 
     if (warp == kConsumers / 32) {
         // ---------------- producer: one lane streams row tiles into the ring
@@ -233,14 +252,15 @@ cyc_encode_ring_kernel(const float* __restrict__ G, float2* __restrict__ Z, int6
             uint32_t cnt = 0;
             bool ok = true;
             for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
-                const int64_t c0 = tile * kTile;
-                const uint32_t bytes = (uint32_t)(((len - c0) < kTile ? (len - c0) : kTile) * 4);
+                const int64_t c0 = tile * kTileCoords;
+                const uint32_t bytes = (uint32_t)(((len - c0) < kTileCoords ? (len - c0) : kTileCoords) * 4);
                 const float* src = G + c0;
                 for (int r = 0; r < n; ++r, ++cnt, src += ldg) {
                     const uint32_t st = cnt & (kStages - 1), par = (cnt / kStages) & 1;
                     if (!mbar_wait(empty0 + 8 * st, par ^ 1)) { ok = false; break; }
-                    mbar_expect_tx(full0 + 8 * st, bytes);
+                    mbar_expect_tx(full0 + 8 * st, PACKED ? 2 * bytes : bytes);
                     bulk_g2s(smem_u32(ring + st * kTile), src, bytes, full0 + 8 * st);
+                    if (PACKED) bulk_g2s(smem_u32(ring + st * kTile + kTile / 2), src + half, bytes, full0 + 8 * st);
                 }
             }
             if (!ok) {
@@ -260,22 +280,22 @@ cyc_encode_ring_kernel(const float* __restrict__ G, float2* __restrict__ Z, int6
     RingState rs;
     rs.full0 = full0; rs.empty0 = empty0; rs.st = 0; rs.par = 0;
     rs.pend_bar = 0; rs.pend_bits = 0; rs.pending = false;
-    const float* ring_t = ring + tid * kVec;
+    const float* ring_t = ring + tid * kPerThread;
     float* stash_t = stash + tid * kVec;
     const int total = n + 2 * S;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const int64_t c0 = tile * kTile;
-        const bool active = c0 + tid * kVec < len;
-        float2* zcol = Z + c0 + tid * kVec;
+        const int64_t c0 = tile * kTileCoords;
+        const bool active = c0 + tid * kPerThread < len;
+        float2* zcol = Z + c0 + tid * kPerThread;
         bool ok = true;
         int v0 = 0;
         if (n >= SL && S > 0) {
-            ok = encode_chunk<S, 0>(w, rs, 0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
+            ok = encode_chunk<S, 0, PACKED>(w, rs, 0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
             for (v0 = SL; ok && v0 + SL <= n; v0 += SL)
-                ok = encode_chunk<S, 1>(w, rs, v0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
+                ok = encode_chunk<S, 1, PACKED>(w, rs, v0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
         }
         for (; ok && v0 < total; v0 += SL)
-            ok = encode_chunk<S, 2>(w, rs, v0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
+            ok = encode_chunk<S, 2, PACKED>(w, rs, v0, n, ring_t, stash_t, zcol, ldz, active, lane, taps, taps64, ph64);
         if (!ok) {
             atomicExch(err, 2);
             return;
@@ -289,33 +309,44 @@ cyc_encode_ring_kernel(const float* __restrict__ G, float2* __restrict__ Z, int6
 }
 
 // Any s, any length / alignment: one coordinate per thread, rows re-read through the caches,
-// fp64 accumulation throughout.
+// fp64 accumulation throughout.  half > 0: packed mode (len complex coordinates; the imaginary
+// parts come from G[r][half + i], zero beyond d_real).
 __global__ void __launch_bounds__(kGenericThreads)
 cyc_encode_generic_kernel(const float* __restrict__ G, float2* __restrict__ Z, int64_t len, int64_t ldg, int64_t ldz,
-                          int n, int s, const float2* __restrict__ taps, const __grid_constant__ EncodePhase64 ph) {
+                          int64_t half, int64_t d_real, int n, int s, const float2* __restrict__ taps,
+                          const __grid_constant__ EncodePhase64 ph) {
     const int64_t stride = (int64_t)gridDim.x * kGenericThreads;
     for (int64_t i = (int64_t)blockIdx.x * kGenericThreads + threadIdx.x; i < len; i += stride) {
+        const bool has_b = half > 0 && half + i < d_real;
         for (int j = 0; j < n; ++j) {
-            double ar = 0.0, ai = 0.0;
+            double ar = 0.0, ai = 0.0, br = 0.0, bi = 0.0;
             for (int t = 0; t <= 2 * s; ++t) {
                 int r = j - t;
                 if (r < 0) r += n;
-                const double g = (double)G[(int64_t)r * ldg + i];
                 const float2 c = taps[t];
+                const double g = (double)G[(int64_t)r * ldg + i];
                 ar = fma((double)c.x, g, ar);
                 ai = fma((double)c.y, g, ai);
+                if (has_b) {
+                    const double gb = (double)G[(int64_t)r * ldg + half + i];
+                    br = fma((double)c.x, gb, br);
+                    bi = fma((double)c.y, gb, bi);
+                }
             }
             const double2 rot = ph.phase[j];
-            Z[(int64_t)j * ldz + i] = make_float2((float)fma(ar, rot.x, -ai * rot.y), (float)fma(ar, rot.y, ai * rot.x));
+            const double xr = fma(ar, rot.x, -ai * rot.y), xi = fma(ar, rot.y, ai * rot.x);
+            const double yr = fma(br, rot.x, -bi * rot.y), yi = fma(br, rot.y, bi * rot.x);
+            Z[(int64_t)j * ldz + i] = make_float2((float)(xr - yi), (float)(xi + yr));
         }
     }
 }
 
-template <int S>
-int launch_ring(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz, cudaStream_t st) {
+template <int S, bool PACKED>
+int launch_ring(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz, int64_t half,
+                cudaStream_t st) {
     constexpr int NSTASH = S > 0 ? 2 * S : 1;
     const size_t smem = sizeof(float) * kTile * (kStages + NSTASH) + 16 * kStages;
-    auto kern = cyc_encode_ring_kernel<S>;
+    auto kern = cyc_encode_ring_kernel<S, PACKED>;
     static bool configured[64] = {};
     int dev = p->device;
     if (dev < 0 || dev >= 64) dev = 0;
@@ -326,40 +357,51 @@ int launch_ring(const draco_plan* p, const float* G, float2* Z, int64_t len, int
     int per_sm = 1;
     DRACO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kRingThreads, smem));
     if (per_sm < 1) per_sm = 1;
-    const int64_t ntiles = (len + kTile - 1) / kTile;
+    constexpr int kTileCoords = PACKED ? kTile / 2 : kTile;
+    const int64_t ntiles = (len + kTileCoords - 1) / kTileCoords;
     int64_t grid = (int64_t)p->sm_count * per_sm;
     if (grid > ntiles) grid = ntiles;
     if (grid < 1) grid = 1;
-    kern<<<(int)grid, kRingThreads, smem, st>>>(G, Z, len, ldg, ldz, p->n, p->taps, p->taps64, p->phase64,
+    kern<<<(int)grid, kRingThreads, smem, st>>>(G, Z, len, ldg, ldz, half, p->n, p->taps, p->taps64, p->phase64,
                                                &p->info_dev->internal_error);
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }
 
+template <bool PACKED>
+int launch_ring_any(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz, int64_t half,
+                    cudaStream_t st) {
+    switch (p->s) {
+        case 0: return launch_ring<0, PACKED>(p, G, Z, len, ldg, ldz, half, st);
+        case 1: return launch_ring<1, PACKED>(p, G, Z, len, ldg, ldz, half, st);
+        case 2: return launch_ring<2, PACKED>(p, G, Z, len, ldg, ldz, half, st);
+        case 3: return launch_ring<3, PACKED>(p, G, Z, len, ldg, ldz, half, st);
+        case 4: return launch_ring<4, PACKED>(p, G, Z, len, ldg, ldz, half, st);
+        case 5: return launch_ring<5, PACKED>(p, G, Z, len, ldg, ldz, half, st);
+        case 6: return launch_ring<6, PACKED>(p, G, Z, len, ldg, ldz, half, st);
+        default: return launch_ring<7, PACKED>(p, G, Z, len, ldg, ldz, half, st);
+    }
+}
+
 }  // namespace
 
+// half == 0: Z[j][i], i < len, from G[.][i].  half > 0 (packed): Z[j][i], i < len complex coordinates,
+// from G[.][i] (real parts) and G[.][half + i] (imaginary parts, zero for half + i >= d_real).
 int launch_cyc_encode(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz,
-                      cudaStream_t st) {
-    // the ring kernel needs 16-byte aligned row tiles: every row start and tile start a multiple of 4 floats
-    const bool fast = (len % 4 == 0) && (ldg % 4 == 0) && (ldz % 2 == 0) && p->s <= 7;
-    if (fast) {
-        switch (p->s) {
-            case 0: return launch_ring<0>(p, G, Z, len, ldg, ldz, st);
-            case 1: return launch_ring<1>(p, G, Z, len, ldg, ldz, st);
-            case 2: return launch_ring<2>(p, G, Z, len, ldg, ldz, st);
-            case 3: return launch_ring<3>(p, G, Z, len, ldg, ldz, st);
-            case 4: return launch_ring<4>(p, G, Z, len, ldg, ldz, st);
-            case 5: return launch_ring<5>(p, G, Z, len, ldg, ldz, st);
-            case 6: return launch_ring<6>(p, G, Z, len, ldg, ldz, st);
-            default: return launch_ring<7>(p, G, Z, len, ldg, ldz, st);
-        }
-    }
+                      int64_t half, int64_t d_real, cudaStream_t st) {
+    // the ring kernel needs 16-byte aligned row slices: row starts, tile starts and the half offset multiples of 4 floats
+    const bool packed = half > 0;
+    bool fast = (ldg % 4 == 0) && (ldz % 2 == 0) && p->s <= 7;
+    if (packed) fast = fast && (len % 4 == 0) && (half % 4 == 0) && (half + len <= d_real);
+    else fast = fast && (len % 4 == 0);
+    if (fast) return packed ? launch_ring_any<true>(p, G, Z, len, ldg, ldz, half, st)
+                            : launch_ring_any<false>(p, G, Z, len, ldg, ldz, 0, st);
     int64_t want = (len + kGenericThreads - 1) / kGenericThreads;
     const int64_t cap = (int64_t)p->sm_count * 16;
     if (want > cap) want = cap;
     if (want < 1) want = 1;
-    cyc_encode_generic_kernel<<<(int)want, kGenericThreads, 0, st>>>(G, Z, len, ldg, ldz, p->n, p->s, p->taps_full_dev,
-                                                                     p->phase64);
+    cyc_encode_generic_kernel<<<(int)want, kGenericThreads, 0, st>>>(G, Z, len, ldg, ldz, half, d_real, p->n, p->s,
+                                                                     p->taps_full_dev, p->phase64);
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }

@@ -13,10 +13,12 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kUnroll = 8;
 
-template <bool VEC2>
+// PACKED: the vectors carry two gradient coordinates per complex entry (Section 3, last
+// paragraph): u[i] = Re(u-hat_i), u[len + i] = Im(u-hat_i) for len + i < d_packed.
+template <bool VEC2, bool PACKED>
 __global__ void __launch_bounds__(kThreads)
 cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const CycDevice* __restrict__ cd,
-                   const DeviceInfo* __restrict__ info, float* __restrict__ u) {
+                   const DeviceInfo* __restrict__ info, float* __restrict__ u, int64_t d_packed) {
     __shared__ double2 bs[kMaxN];
     __shared__ int rows[kMaxN];
     const int count = info->n_active;
@@ -30,7 +32,7 @@ cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const 
         const int64_t nvec = len / 2;
         for (int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x; v < nvec; v += stride) {
             const float2* col = R + v * 2;
-            double a0 = 0.0, a1 = 0.0;
+            double a0 = 0.0, a1 = 0.0, i0 = 0.0, i1 = 0.0;
             for (int k0 = 0; k0 < count; k0 += kUnroll) {
                 float4 x[kUnroll];
 #pragma unroll
@@ -40,41 +42,61 @@ cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const 
                 for (int q = 0; q < kUnroll; ++q)
                     if (k0 + q < count) {
                         const double2 b = bs[k0 + q];
-                        a0 = fma(b.x, (double)x[q].x, a0);
-                        a0 = fma(-b.y, (double)x[q].y, a0);
-                        a1 = fma(b.x, (double)x[q].z, a1);
-                        a1 = fma(-b.y, (double)x[q].w, a1);
+                        const double xr0 = (double)x[q].x, xi0 = (double)x[q].y, xr1 = (double)x[q].z, xi1 = (double)x[q].w;
+                        a0 = fma(b.x, xr0, a0);
+                        a0 = fma(-b.y, xi0, a0);
+                        a1 = fma(b.x, xr1, a1);
+                        a1 = fma(-b.y, xi1, a1);
+                        if (PACKED) {
+                            i0 = fma(b.x, xi0, i0);
+                            i0 = fma(b.y, xr0, i0);
+                            i1 = fma(b.x, xi1, i1);
+                            i1 = fma(b.y, xr1, i1);
+                        }
                     }
             }
             __stcs(reinterpret_cast<float2*>(u + v * 2), make_float2((float)a0, (float)a1));
+            if (PACKED) __stcs(reinterpret_cast<float2*>(u + len + v * 2), make_float2((float)i0, (float)i1));
         }
     } else {
         for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < len; i += stride) {
-            double a0 = 0.0;
+            double a0 = 0.0, i0 = 0.0;
             for (int k = 0; k < count; ++k) {
                 const float2 x = __ldcs(R + (int64_t)rows[k] * ld + i);
                 const double2 b = bs[k];
                 a0 = fma(b.x, (double)x.x, a0);
                 a0 = fma(-b.y, (double)x.y, a0);
+                if (PACKED) {
+                    i0 = fma(b.x, (double)x.y, i0);
+                    i0 = fma(b.y, (double)x.x, i0);
+                }
             }
             u[i] = (float)a0;
+            if (PACKED && len + i < d_packed) u[len + i] = (float)i0;
         }
     }
 }
 
 }  // namespace
 
-int launch_cyc_recover(draco_plan* p, const float2* R, int64_t len, int64_t ld, float* u, cudaStream_t st) {
-    const bool vec2 = (len % 2 == 0) && (ld % 2 == 0);
+int launch_cyc_recover(draco_plan* p, const float2* R, int64_t len, int64_t ld, float* u, int64_t d_packed,
+                       cudaStream_t st) {
+    const bool packed = d_packed > 0;
+    // 64-bit stores of u need len even; in packed mode the second half starts at u + len and must cover it fully
+    const bool vec2 = (len % 2 == 0) && (ld % 2 == 0) && (!packed || d_packed == 2 * len);
     const int64_t nvec = vec2 ? len / 2 : len;
     int64_t want = (nvec + kThreads - 1) / kThreads;
     const int64_t cap = (int64_t)p->sm_count * 16;
     if (want > cap) want = cap;
     if (want < 1) want = 1;
-    if (vec2)
-        cyc_recover_kernel<true><<<(int)want, kThreads, 0, st>>>(R, len, ld, p->cyc_dev, p->info_dev, u);
-    else
-        cyc_recover_kernel<false><<<(int)want, kThreads, 0, st>>>(R, len, ld, p->cyc_dev, p->info_dev, u);
+#define DRACO_REC(V2, PK) \
+    cyc_recover_kernel<V2, PK><<<(int)want, kThreads, 0, st>>>(R, len, ld, p->cyc_dev, p->info_dev, u, d_packed)
+    if (vec2) {
+        if (packed) DRACO_REC(true, true); else DRACO_REC(true, false);
+    } else {
+        if (packed) DRACO_REC(false, true); else DRACO_REC(false, false);
+    }
+#undef DRACO_REC
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }

@@ -26,6 +26,11 @@ namespace {
 typedef std::complex<long double> cld;
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool is_cyc(const draco_plan* p) { return p->code == DRACO_CYC || p->code == DRACO_CYC_PACKED; }
+inline bool is_packed(const draco_plan* p) { return p->code == DRACO_CYC_PACKED; }
+// entries per worker vector: d, or ceil(d / 2) complex entries in packed mode
+inline int64_t vec_len(const draco_plan* p) { return is_packed(p) ? (p->d + 1) / 2 : p->d; }
+inline int64_t half_off(const draco_plan* p) { return is_packed(p) ? (p->d + 1) / 2 : 0; }
 
 cld root_of_unity(int n, long long e) {
     const long double pi = 3.141592653589793238462643383279502884L;
@@ -127,7 +132,7 @@ int draco_plan_create(int n, int s, int64_t d, int code, draco_plan** out) {
     if (!out) return DRACO_EINVAL;
     *out = nullptr;
     if (n < 1 || n > DRACO_MAX_N || s < 0 || 2 * s + 1 > n || d < 1) return DRACO_EINVAL;
-    if (code != DRACO_REP && code != DRACO_CYC) return DRACO_EINVAL;
+    if (code != DRACO_REP && code != DRACO_CYC && code != DRACO_CYC_PACKED) return DRACO_EINVAL;
     draco_plan* p = new (std::nothrow) draco_plan();
     if (!p) return DRACO_ENOMEM;
     memset(p, 0, sizeof(*p));
@@ -199,7 +204,7 @@ int draco_groups(const draco_plan* plan, int* first, int* size) {
 }
 
 int draco_cyc_W(const draco_plan* plan, double* W_host) {
-    if (!plan || plan->code != DRACO_CYC || !W_host) return DRACO_EINVAL;
+    if (!plan || !is_cyc(plan) || !W_host) return DRACO_EINVAL;
     // stored by rows of the construction (row j = node j's allocation); hand out W itself
     memcpy(W_host, plan->W_host, sizeof(double) * 2 * (size_t)plan->n * plan->n);
     return DRACO_OK;
@@ -209,7 +214,7 @@ int draco_encode(const draco_plan* plan, const float* G, void* Z, void* stream) 
     if (!plan || !G || !Z || !aligned16(G) || !aligned16(Z)) return DRACO_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     if (plan->code == DRACO_REP) return launch_rep_encode(plan, G, (float*)Z, plan->d, plan->d, plan->d, st);
-    return launch_cyc_encode(plan, G, (float2*)Z, plan->d, plan->d, plan->d, st);
+    return launch_cyc_encode(plan, G, (float2*)Z, vec_len(plan), plan->d, vec_len(plan), half_off(plan), plan->d, st);
 }
 
 int draco_rep_vote(draco_plan* plan, const void* R, float* u, float* maj, uint8_t* flags, void* stream) {
@@ -218,16 +223,16 @@ int draco_rep_vote(draco_plan* plan, const void* R, float* u, float* maj, uint8_
 }
 
 int draco_cyc_project(draco_plan* plan, const void* R, const float* f, double* e, void* stream) {
-    if (!plan || plan->code != DRACO_CYC || !R || !f || !e || !aligned16(R) || !aligned16(f) || !aligned16(e))
+    if (!plan || !is_cyc(plan) || !R || !f || !e || !aligned16(R) || !aligned16(f) || !aligned16(e))
         return DRACO_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
-    int rc = launch_cyc_project(plan, (const float2*)R, f, plan->d, plan->d, false, st);
+    int rc = launch_cyc_project(plan, (const float2*)R, f, vec_len(plan), vec_len(plan), false, st);
     if (rc != DRACO_OK) return rc;
     return launch_cyc_project_finish(plan, (double2*)e, st);
 }
 
 int draco_cyc_locate_from_projection(draco_plan* plan, const double* e, uint8_t* flags, void* stream) {
-    if (!plan || plan->code != DRACO_CYC || !e || !flags || !aligned16(e)) return DRACO_EINVAL;
+    if (!plan || !is_cyc(plan) || !e || !flags || !aligned16(e)) return DRACO_EINVAL;
     return launch_cyc_solve(plan, (const double2*)e, flags, (cudaStream_t)stream);
 }
 
@@ -237,7 +242,7 @@ int draco_locate(draco_plan* plan, const void* R, const float* f, uint8_t* flags
     if (plan->code == DRACO_REP)
         return launch_rep_vote(plan, (const float*)R, plan->d, plan->d, nullptr, nullptr, flags, true, st);
     if (!f || !aligned16(f)) return DRACO_EINVAL;
-    int rc = launch_cyc_project(plan, (const float2*)R, f, plan->d, plan->d, false, st);
+    int rc = launch_cyc_project(plan, (const float2*)R, f, vec_len(plan), vec_len(plan), false, st);
     if (rc != DRACO_OK) return rc;
     return launch_cyc_solve(plan, nullptr, flags, st);
 }
@@ -250,7 +255,7 @@ int draco_decode(draco_plan* plan, const void* R, const uint8_t* flags, float* u
     if (!flags) return DRACO_EINVAL;
     int rc = launch_cyc_decode_vector(plan, flags, st);
     if (rc != DRACO_OK) return rc;
-    return launch_cyc_recover(plan, (const float2*)R, plan->d, plan->d, u, st);
+    return launch_cyc_recover(plan, (const float2*)R, vec_len(plan), vec_len(plan), u, is_packed(plan) ? plan->d : 0, st);
 }
 
 int draco_locate_decode(draco_plan* plan, const void* R, const float* f, uint8_t* flags, float* u, void* stream) {
@@ -264,7 +269,7 @@ int draco_locate_decode(draco_plan* plan, const void* R, const float* f, uint8_t
 }
 
 int draco_cyc_decode_vector(draco_plan* plan, double* b_host, void* stream) {
-    if (!plan || plan->code != DRACO_CYC || !b_host) return DRACO_EINVAL;
+    if (!plan || !is_cyc(plan) || !b_host) return DRACO_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     DRACO_CUDA(cudaMemcpyAsync(b_host, plan->cyc_dev->b, sizeof(double2) * plan->n, cudaMemcpyDeviceToHost, st));
     DRACO_CUDA(cudaStreamSynchronize(st));
@@ -296,7 +301,7 @@ int draco_generate(float* out, int rows, int64_t len, int row0, float mean, floa
 
 static int corrupt_range(const draco_plan* plan, void* R, int64_t c0, int64_t len, int64_t ld, const int* adv_idx,
                          const int* adv_model, const float* adv_param, int n_adv, uint64_t seed, cudaStream_t st) {
-    const bool cplx = plan->code == DRACO_CYC;
+    const bool cplx = is_cyc(plan);
     const int64_t per = cplx ? 2 : 1;
     for (int a = 0; a < n_adv; ++a) {
         const int j = adv_idx[a];
@@ -312,7 +317,8 @@ static int corrupt_range(const draco_plan* plan, void* R, int64_t c0, int64_t le
 int draco_corrupt(const draco_plan* plan, void* R, const int* adv_idx, const int* adv_model, const float* adv_param,
                   int n_adv, uint64_t seed, void* stream) {
     if (!plan || !R || n_adv < 0 || (n_adv > 0 && (!adv_idx || !adv_model || !adv_param))) return DRACO_EINVAL;
-    return corrupt_range(plan, R, 0, plan->d, plan->d, adv_idx, adv_model, adv_param, n_adv, seed, (cudaStream_t)stream);
+    return corrupt_range(plan, R, 0, vec_len(plan), vec_len(plan), adv_idx, adv_model, adv_param, n_adv, seed,
+                         (cudaStream_t)stream);
 }
 
 int draco_pipeline_host(draco_plan* plan, const float* G_host, const float* f_host, const int* adv_idx,
@@ -320,35 +326,46 @@ int draco_pipeline_host(draco_plan* plan, const float* G_host, const float* f_ho
                         float* u_host, uint8_t* flags_host, draco_info* info) {
     if (!plan || !G_host || !Z || !u_host || !flags_host || !aligned16(Z)) return DRACO_EINVAL;
     if (n_adv < 0 || (n_adv > 0 && (!adv_idx || !adv_model || !adv_param))) return DRACO_EINVAL;
-    const bool cyc = plan->code == DRACO_CYC;
+    const bool cyc = is_cyc(plan), packed = is_packed(plan);
     if (cyc && !f_host) return DRACO_EINVAL;
     const int n = plan->n;
     const int64_t d = plan->d;
+    const int64_t vlen = vec_len(plan);              // entries per worker vector (complex entries when packed)
     // column chunk: about 256 MB of G per copy, a multiple of the projection tile
     int64_t chunk = ((int64_t)64 << 20) / n;
-    chunk = (chunk / kProjectTile) * kProjectTile;
-    if (chunk < kProjectTile) chunk = kProjectTile;
-    if (chunk > d) chunk = d;
+    chunk = (chunk / (2 * kProjectTile)) * (2 * kProjectTile);
+    if (chunk < 2 * kProjectTile) chunk = 2 * kProjectTile;
     if (!plan->stage_dev) {
         DRACO_CUDA(cudaMalloc(&plan->stage_dev, sizeof(float) * (size_t)n * chunk));
         plan->stage_chunk = chunk;
     }
     if (!plan->u_dev) DRACO_CUDA(cudaMalloc(&plan->u_dev, sizeof(float) * (size_t)d));
-    if (cyc && !plan->f_dev) DRACO_CUDA(cudaMalloc(&plan->f_dev, sizeof(float) * (size_t)d));
+    if (cyc && !plan->f_dev) DRACO_CUDA(cudaMalloc(&plan->f_dev, sizeof(float) * (size_t)vlen));
     chunk = plan->stage_chunk;
+    const int64_t step = packed ? chunk / 2 : chunk;   // vector entries per chunk
     cudaStream_t st = 0;
-    if (cyc) DRACO_CUDA(cudaMemcpyAsync(plan->f_dev, f_host, sizeof(float) * (size_t)d, cudaMemcpyHostToDevice, st));
+    if (cyc) DRACO_CUDA(cudaMemcpyAsync(plan->f_dev, f_host, sizeof(float) * (size_t)vlen, cudaMemcpyHostToDevice, st));
     bool first = true;
-    for (int64_t c0 = 0; c0 < d; c0 += chunk) {
-        const int64_t len = (d - c0) < chunk ? (d - c0) : chunk;
+    for (int64_t c0 = 0; c0 < vlen; c0 += step) {
+        const int64_t len = (vlen - c0) < step ? (vlen - c0) : step;
         DRACO_CUDA(cudaMemcpy2DAsync(plan->stage_dev, sizeof(float) * (size_t)chunk, G_host + c0, sizeof(float) * (size_t)d,
                                      sizeof(float) * (size_t)len, n, cudaMemcpyHostToDevice, st));
         int rc;
         if (cyc) {
+            int64_t half = 0, d_stage = len;
+            if (packed) {                              // second half of the gradient next to the first in the stage
+                const int64_t len_b = (d - vlen - c0) < len ? (d - vlen - c0) : len;
+                if (len_b > 0)
+                    DRACO_CUDA(cudaMemcpy2DAsync(plan->stage_dev + step, sizeof(float) * (size_t)chunk, G_host + vlen + c0,
+                                                 sizeof(float) * (size_t)d, sizeof(float) * (size_t)len_b, n,
+                                                 cudaMemcpyHostToDevice, st));
+                half = step;
+                d_stage = step + (len_b > 0 ? len_b : 0);
+            }
             float2* Zc = (float2*)Z + c0;
-            rc = launch_cyc_encode(plan, plan->stage_dev, Zc, len, chunk, d, st);
-            if (rc == DRACO_OK) rc = corrupt_range(plan, Z, c0, len, d, adv_idx, adv_model, adv_param, n_adv, adv_seed, st);
-            if (rc == DRACO_OK) rc = launch_cyc_project(plan, Zc, plan->f_dev + c0, len, d, !first, st);
+            rc = launch_cyc_encode(plan, plan->stage_dev, Zc, len, chunk, vlen, half, d_stage, st);
+            if (rc == DRACO_OK) rc = corrupt_range(plan, Z, c0, len, vlen, adv_idx, adv_model, adv_param, n_adv, adv_seed, st);
+            if (rc == DRACO_OK) rc = launch_cyc_project(plan, Zc, plan->f_dev + c0, len, vlen, !first, st);
         } else {
             float* Zc = (float*)Z + c0;
             rc = launch_rep_encode(plan, plan->stage_dev, Zc, len, chunk, d, st);
@@ -361,7 +378,7 @@ int draco_pipeline_host(draco_plan* plan, const float* G_host, const float* f_ho
     if (cyc) {
         rc = launch_cyc_solve(plan, nullptr, nullptr, st);
         if (rc == DRACO_OK) rc = launch_cyc_decode_vector(plan, plan->flags_dev, st);
-        if (rc == DRACO_OK) rc = launch_cyc_recover(plan, (const float2*)Z, d, d, plan->u_dev, st);
+        if (rc == DRACO_OK) rc = launch_cyc_recover(plan, (const float2*)Z, vlen, vlen, plan->u_dev, packed ? d : 0, st);
     } else {
         rc = launch_rep_vote(plan, (const float*)Z, d, d, plan->u_dev, nullptr, nullptr, true, st);
     }

@@ -282,3 +282,124 @@ def test_full_size_decode_on_generated_R_sampled():
     Rs = di.complex_rows(555, n, d, idx=idx)
     uo = orc.cyc_decode(Rs, n, s, flags.astype(bool))
     assert normwise(host(u[idx]), uo) <= 1e-6
+
+
+# ------------------------------------------------------------------ packed transport (Section 3, last paragraph)
+# (n, s, d): d % 8 == 0 takes the ring kernel and 64-bit stores; the others the generic paths (odd d pads the last imaginary part)
+PACKED_SHAPES = [(15, 2, 100_000), (45, 5, 24_592), (45, 3, 6152), (15, 2, 1001), (9, 1, 6), (15, 7, 4100), (20, 8, 1032)]
+
+
+def _packed_plan(n, s, d):
+    import paper_1803_09877_b200 as dr
+    return dr, dr.Plan(n, s, d, dr.CYC_PACKED)
+
+
+@pytest.mark.parametrize("n,s,d", PACKED_SHAPES)
+def test_packed_encode_parity(n, s, d):
+    dr, plan = _packed_plan(n, s, d)
+    h = (d + 1) // 2
+    G = di.gradient_rows(0xD2AC0 + n + s, n, d)
+    Z = torch.empty((n, 2 * h), dtype=torch.float32, device="cuda")
+    plan.encode(dev(G), Z)
+    torch.cuda.synchronize()
+    Zg = host(Z, complex64=True)
+    Zo = orc.cyc_encode_packed(G, n, s, dtype=np.complex128)
+    assert Zg.shape == Zo.shape == (n, h)
+    for j in range(n):
+        assert np.abs(Zg[j] - Zo[j]).max() <= 1e-6 * np.abs(Zo[j]).max(), j
+
+
+@pytest.mark.parametrize("n,s,d", PACKED_SHAPES)
+def test_packed_locate_decode_parity_and_exact_sum(n, s, d):
+    dr, plan = _packed_plan(n, s, d)
+    h = (d + 1) // 2
+    seed = 23 * n + s
+    G = di.gradient_rows(seed, n, d)
+    R = orc.cyc_encode_packed(G, n, s)                     # complex64 worker vectors of h entries
+    adv = di.choose_adversaries(seed + 1, n, s)
+    di.apply_adversaries(R, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2)
+    f = di.projection_vector(seed + 3, h)
+    want = orc.cyc_locate(R, f, n, s)
+    assert sorted(np.flatnonzero(want["flags"])) == adv.tolist() and want["margin"] > 10
+    Rd, fd = dev(R), dev(f)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    u = torch.full((d,), float("nan"), dtype=torch.float32, device="cuda")
+    plan.locate_decode(Rd, fd, flags, u)
+    info = plan.info()
+    np.testing.assert_array_equal(host(flags).astype(bool), want["flags"])
+    assert info["status"] == 0 and info["locator_rank"] == s
+    uo = orc.cyc_decode_packed(R, n, s, want["flags"], d)
+    assert uo.shape == (d,)
+    assert normwise(host(u), uo) <= 1e-6                    # identical R, identical flags
+    # whole path on the device against G 1_P
+    Z = torch.empty((n, 2 * h), dtype=torch.float32, device="cuda")
+    plan.encode(dev(G), Z)
+    plan.corrupt(Z, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2)
+    plan.locate_decode(Z, fd, flags, u)
+    torch.cuda.synchronize()
+    assert sorted(np.flatnonzero(host(flags))) == adv.tolist()
+    exact = G.astype(np.float64).sum(axis=0)
+    floor = normwise(uo, exact)
+    assert normwise(host(u), exact) <= max(1e-4 if n <= 21 else 0.0, 2.0 * floor + 1e-6)
+
+
+def test_packed_host_pipeline():
+    n, s, d = 15, 2, 300_008
+    dr, plan = _packed_plan(n, s, d)
+    h = d // 2
+    seed = 5151
+    G = di.gradient_rows(seed, n, d)
+    f = di.projection_vector(seed + 3, h)
+    adv = di.choose_adversaries(seed + 1, n, s)
+    Z = torch.empty((n, 2 * h), dtype=torch.float32, device="cuda")
+    u_host = np.empty(d, dtype=np.float32)
+    flags_host = np.empty(n, dtype=np.uint8)
+    info = plan.pipeline_host(G.ctypes.data, f.ctypes.data, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed + 2, Z,
+                              u_host.ctypes.data, flags_host.ctypes.data)
+    assert info["status"] == 0 and sorted(np.flatnonzero(flags_host)) == adv.tolist()
+    assert normwise(u_host, G.astype(np.float64).sum(axis=0)) <= 1e-4
+    Z2 = torch.empty_like(Z)
+    plan.encode(dev(G), Z2)
+    plan.corrupt(Z2, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2)
+    torch.cuda.synchronize()
+    assert torch.equal(Z, Z2)
+
+
+def test_packed_full_size_resnet152_sampled():
+    """Packed transport at n = 45, s = 5, d = 60.2 M: 30.1 M complex entries per worker (10.8 GB instead of 21.7 GB)."""
+    import paper_1803_09877_b200 as dr
+    n, s, d = 45, 5, 60_200_000
+    h = d // 2
+    plan = dr.Plan(n, s, d, dr.CYC_PACKED)
+    seed = 0xD2AC0 + 6
+    G = torch.empty((n, d), dtype=torch.float32, device="cuda")
+    dr.generate(G, n, d, seed=seed)
+    f = torch.empty(h, dtype=torch.float32, device="cuda")
+    dr.generate(f, 1, h, mean=1.0, std=1.0, seed=seed + 3)
+    Z = torch.empty((n, 2 * h), dtype=torch.float32, device="cuda")
+    plan.encode(G, Z)
+    adv = di.choose_adversaries(seed + 1, n, s)
+    plan.corrupt(Z, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.locate_decode(Z, f, flags, u)
+    assert plan.info()["status"] == 0
+    assert sorted(np.flatnonzero(host(flags))) == adv.tolist()
+    rng = np.random.default_rng(4)
+    ci = np.unique(np.concatenate([np.arange(2048), np.arange(h - 2048, h), rng.integers(0, h, 50_000)]))
+    both = np.concatenate([ci, h + ci])
+    Gs = di.gradient_rows(seed, n, d, idx=both)
+    np.testing.assert_array_equal(host(G[:, both]), Gs)
+    exact = Gs.astype(np.float64).sum(axis=0)
+    Ghat = Gs[:, : len(ci)].astype(np.float64) + 1j * Gs[:, len(ci):].astype(np.float64)
+    Zo = orc.cyc_W(n, s).T @ Ghat
+    Zg = host(Z.view(n, h, 2)[:, ci, :].contiguous().view(n, -1), complex64=True)
+    for j in np.setdiff1d(np.arange(n), adv):
+        assert np.abs(Zg[j] - Zo[j]).max() <= 1e-6 * np.abs(Zo[j]).max()
+    want_flags = np.zeros(n, dtype=bool)
+    want_flags[adv] = True
+    Ro = Zo.astype(np.complex64)
+    di.apply_adversaries(Ro, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2, idx=ci)
+    uhat = orc.cyc_recover(Ro, orc.cyc_decode_vector(n, s, want_flags))
+    floor = normwise(np.concatenate([uhat.real, uhat.imag]), exact)
+    assert normwise(host(u[both]), exact) <= 2.0 * floor + 1e-6

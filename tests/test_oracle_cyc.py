@@ -221,3 +221,37 @@ def test_complex64_transport_floor():
         assert list(np.flatnonzero(out["flags"])) == adv.tolist()
         err = np.abs(out["u"] - _exact_sum(G)).max() / np.abs(_exact_sum(G)).max()
         assert lo <= err <= hi, err
+
+
+@pytest.mark.parametrize("d", [1, 2, 7, 8, 33])
+def test_packing_round_trip_and_sum(d):
+    n = 5
+    G = di.gradient_rows(81, n, d)
+    Gh = orc.cyc_pack(G)
+    assert Gh.shape == (n, (d + 1) // 2)
+    for k in range(n):
+        np.testing.assert_array_equal(orc.cyc_unpack(Gh[k], d), G[k].astype(np.float64))
+    np.testing.assert_array_equal(orc.cyc_unpack(Gh.sum(axis=0), d), G.astype(np.float64).sum(axis=0))
+    if d >= 7:   # the literal "Re + Im" of the text is not the gradient sum
+        literal = Gh.sum(axis=0).real + Gh.sum(axis=0).imag
+        assert literal.shape[0] != d or np.abs(literal - G.astype(np.float64).sum(axis=0)).max() > 1e-3
+
+
+@pytest.mark.parametrize("n,s,d", [(4, 1, 9), (7, 2, 16), (9, 2, 31), (15, 2, 40)])
+def test_packed_pipeline_corrects_every_placement(n, s, d):
+    """Definition 2 through the packed transport: half the complex coordinates, same guarantee."""
+    G = di.gradient_rows(91, n, d)
+    Z = orc.cyc_encode_packed(G, n, s, dtype=np.complex128)
+    h = (d + 1) // 2
+    assert Z.shape == (n, h)
+    f = di.projection_vector(92, h)
+    exact = _exact_sum(G)
+    for a in range(s + 1):
+        for placement in itertools.combinations(range(n), a):
+            R = Z.copy()
+            R[list(placement)] *= -100.0
+            loc = orc.cyc_locate(R, f, n, s)
+            assert set(np.flatnonzero(loc["flags"])) == set(placement)
+            u = orc.cyc_decode_packed(R, n, s, loc["flags"], d)
+            assert u.shape == (d,)
+            assert np.abs(u - exact).max() <= 1e-8 * np.abs(exact).max()
