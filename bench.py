@@ -36,6 +36,7 @@ WORKLOADS = {
     # name: (code, n, s, d, gradient std, adversary models, params)
     "cyc_n45_s5_d60.2M": ("cyc", 45, 5, 60_200_000, 1.0, ["revgrad"], [100.0]),
     "rep_n45_s3_d11.7M": ("rep", 45, 3, 11_700_000, 0.1, ["revgrad", "const"], [100.0, 1e4]),
+    "cycp_n45_s5_d60.2M": ("cycp", 45, 5, 60_200_000, 1.0, ["revgrad"], [100.0]),   # packed transport: 30.1 M complex entries
     "cyc_n15_s2_d1M": ("cyc", 15, 2, 1_000_000, 1.0, ["gauss"], [1e3]),
     "rep_n15_s2_d100k": ("rep", 15, 2, 100_000, 1.0, ["revgrad"], [100.0]),
 }
@@ -63,6 +64,10 @@ def adversaries(workload, rank=0):
 
 def algorithmic_bytes(code, n, s, d, n_adv):
     """Bytes each stage must move (per step, one GPU)."""
+    if code == "cycp":
+        h = (d + 1) // 2
+        return {"encode": 4 * n * d + 8 * n * h, "locate": 8 * n * h + 4 * h, "decode": 8 * (n - n_adv) * h + 4 * d,
+                "corrupt": 2 * 8 * n_adv * h, "coded": 8 * n * h}
     if code == "cyc":
         return {"encode": 4 * n * d + 8 * n * d, "locate": 8 * n * d + 4 * d, "decode": 8 * (n - n_adv) * d + 4 * d,
                 "corrupt": 2 * 8 * n_adv * d, "coded": 8 * n * d}
@@ -79,7 +84,13 @@ def oracle_step(workload, d_sample, seed):
     G = di.gradient_rows(seed, n, d, 0.0, std, i0=0, i1=d_sample)
     f = di.projection_vector(seed + 3, d, i0=0, i1=d_sample)
     t0 = time.perf_counter()
-    if code == "cyc":
+    if code == "cycp":         # the sample's own two halves are packed together
+        R = orc.cyc_encode_packed(G, n, s)
+        di.apply_adversaries(R, adv, model, param, seed=seed + 2)
+        out = orc.cyc_locate(R, f[: R.shape[1]], n, s)
+        orc.cyc_decode_packed(R, n, s, out["flags"], d_sample)
+        ok = sorted(np.flatnonzero(out["flags"])) == adv.tolist()
+    elif code == "cyc":
         R = orc.cyc_encode(G, n, s)
         di.apply_adversaries(R, adv, model, param, seed=seed + 2)
         out = orc.cyc_decode_full(R, f, n, s)
@@ -109,7 +120,7 @@ def cpu_baseline(workload, target_seconds=15.0):
     dt, _ = oracle_step(workload, probe, SEED)
     d_sample = int(min(d, max(probe, probe * target_seconds / max(dt, 1e-3))))
     dt, ok = oracle_step(workload, d_sample, SEED)
-    per = 8 if code == "cyc" else 4
+    per = 8 if code == "cyc" else 4                      # coded bytes per gradient coordinate (packed: 8 per 2)
     return {"value": per * n * d_sample / dt / 1e9, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
             "sample": f"first {d_sample} of {d} coordinates, all {n} workers, one pass in {dt:.2f} s "
                       f"(numpy fp64/complex128; flags correct: {ok})"}
@@ -210,9 +221,11 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     workload = args.workload
     code, n, s, d, std, models, params = WORKLOADS[workload]
-    cyc = code == "cyc"
+    cyc = code in ("cyc", "cycp")
+    packed = code == "cycp"
+    vlen = (d + 1) // 2 if packed else d                 # entries per worker vector
     adv, model, param = adversaries(workload)
-    plan = dr.Plan(n, s, d, dr.CYC if cyc else dr.REP)
+    plan = dr.Plan(n, s, d, dr.CYC_PACKED if packed else dr.CYC if cyc else dr.REP)
     stream = torch.cuda.current_stream()
 
     # inputs resident in HBM; rank r holds coordinates [r d, (r+1) d) of a d * world vector
@@ -220,9 +233,9 @@ def run_gpu(args):
     dr.generate(G, n, d, mean=0.0, std=std, seed=SEED + 17 * rank)
     f = None
     if cyc:
-        f = torch.empty(d, dtype=torch.float32, device="cuda")
-        dr.generate(f, 1, d, mean=1.0, std=1.0, seed=SEED + 3 + 17 * rank)
-    Z = torch.empty((n, (2 if cyc else 1) * d), dtype=torch.float32, device="cuda")
+        f = torch.empty(vlen, dtype=torch.float32, device="cuda")
+        dr.generate(f, 1, vlen, mean=1.0, std=1.0, seed=SEED + 3 + 17 * rank)
+    Z = torch.empty((n, (2 if cyc else 1) * vlen), dtype=torch.float32, device="cuda")
     u = torch.empty(d, dtype=torch.float32, device="cuda")
     flags = torch.empty(n, dtype=torch.uint8, device="cuda")
     e = torch.empty(2 * n, dtype=torch.float64, device="cuda")
@@ -289,10 +302,15 @@ def run_gpu(args):
     value = ab["coded"] * world / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak_gbs()
     if cyc:
-        dom, dom_kernel = "encode", f"cyc_encode_kernel<S={s}>"
+        dom, dom_kernel = "encode", f"cyc_encode_ring_kernel<S={s}, packed={str(packed).lower()}>"
     else:
         dom, dom_kernel = "decode", "rep_vote_kernel"
     achieved = ab[dom] / (stage_ms[dom] * 1e-3) / 1e9
+    # DRAM bytes per gradient coordinate of the dominant kernel, from the ncu captures summarised under profiles/
+    # (dram__bytes_read.sum + dram__bytes_write.sum at d = 4 M / 8 M; every byte is touched once, so traffic scales with d).
+    # Valid for n = 45 with the configured s only; null for any other shape.
+    traffic_per_coord = {("cyc", 45, 5): 525.5, ("cycp", 45, 5): 353.7, ("rep", 45, 3): 183.0}.get((code, n, s))
+    traffic = traffic_per_coord * d if traffic_per_coord else None
     stages = {}
     for nm in names:
         if stage_ms[nm] > 0 and ab.get(nm, 0) > 0:
@@ -309,7 +327,7 @@ def run_gpu(args):
         del events
         Gh = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
         Gh.copy_(G)
-        fh = torch.empty(d, dtype=torch.float32, pin_memory=True)
+        fh = torch.empty(vlen, dtype=torch.float32, pin_memory=True)
         if cyc:
             fh.copy_(f)
         uh = torch.empty(d, dtype=torch.float32, pin_memory=True)
@@ -330,21 +348,21 @@ def run_gpu(args):
         if sorted(np.flatnonzero(flh.numpy()).tolist()) != adv.tolist():
             raise SystemExit("host pipeline: flags differ from the planted adversaries")
         e2e = {"value": ab["coded"] * world / dt / 1e9, "unit": UNIT,
-               "h2d_bytes_per_step": 4 * n * d + (4 * d if cyc else 0), "d2h_bytes_per_step": 4 * d + n,
+               "h2d_bytes_per_step": 4 * n * d + (4 * vlen if cyc else 0), "d2h_bytes_per_step": 4 * d + n,
                "ms_per_step": dt * 1e3, "steps": reps}
 
     if rank == 0:
         cb = cpu_baseline(workload) if (world == 1 and not args.no_cpu_baseline) else None
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32 (complex64 vectors; f64 accumulation in locate/decode)"
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32 (complex64 vectors; f64 centre taps, projection sums and recovery)"
                 if cyc else "f32 (u32 bit patterns in the vote)", "data": "synthetic",
                 "config": {"workload": workload, "code": code, "n": n, "s": s, "d_per_gpu": d, "adversaries": len(adv),
                            "adversary_models": models, "l2": "inputs larger than L2 (no flush needed)"
                            if ab["coded"] > 4e8 else "working set near L2 size: not an HBM number",
                            "value_is": "bytes of coded gradients (n d complex64 / fp32) per step / step time"},
                 "roofline": {"bound": "hbm", "kernel": dom_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                             "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                              "algorithmic_bytes_per_launch": ab[dom], "avg_launch_ms": stage_ms[dom]},
                 "stages": stages, "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "cpu_baseline": cb}
         print(json.dumps(line))
