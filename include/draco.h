@@ -134,6 +134,14 @@ int draco_locate(draco_plan* plan, const void* R, const float* f, uint8_t* flags
  */
 int draco_decode(draco_plan* plan, const void* R, const uint8_t* flags, float* u, void* stream);
 
+/*
+ * Decoding fused with the model update of Section 2 (mini-batch SGD, w_k = w_{k-1} - gamma / |S_k| * sum of gradients):
+ * w <- w - scale * D(R) in the decoder's epilogue; u is never written.  w: device [d] fp32, read and written.
+ * Same arguments and arithmetic as draco_decode; each entry of D(R) is rounded to fp32, then one fused multiply-add.
+ * When more than 2 s nodes are flagged (cyclic) D(R) is zero and w is left unchanged.
+ */
+int draco_decode_update(draco_plan* plan, const void* R, const uint8_t* flags, float* w, float scale, void* stream);
+
 /* locate + decode in one call (repetition: one pass over R; cyclic: locate, then decode). */
 int draco_locate_decode(draco_plan* plan, const void* R, const float* f, uint8_t* flags, float* u, void* stream);
 

@@ -56,6 +56,7 @@ _SIGS = {
     "draco_locate": ([_vp, _vp, _vp, _vp, _vp], _i),
     "draco_decode": ([_vp, _vp, _vp, _vp, _vp], _i),
     "draco_locate_decode": ([_vp, _vp, _vp, _vp, _vp, _vp], _i),
+    "draco_decode_update": ([_vp, _vp, _vp, _vp, _f, _vp], _i),
     "draco_rep_vote": ([_vp, _vp, _vp, _vp, _vp, _vp], _i),
     "draco_cyc_project": ([_vp, _vp, _vp, _vp, _vp], _i),
     "draco_cyc_locate_from_projection": ([_vp, _vp, _vp, _vp], _i),
@@ -162,6 +163,9 @@ class Plan:
 
     def decode(self, R, flags, u, stream=None):
         return _check(lib.draco_decode(self._h, _ptr(R), _ptr(flags), _ptr(u), _stream(stream)))
+
+    def decode_update(self, R, flags, w, scale: float, stream=None):
+        return _check(lib.draco_decode_update(self._h, _ptr(R), _ptr(flags), _ptr(w), scale, _stream(stream)))
 
     def locate_decode(self, R, f, flags, u, stream=None):
         return _check(lib.draco_locate_decode(self._h, _ptr(R), _ptr(f), _ptr(flags), _ptr(u), _stream(stream)))

@@ -18,7 +18,8 @@ constexpr int kUnroll = 8;
 template <bool VEC2, bool PACKED>
 __global__ void __launch_bounds__(kThreads)
 cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const CycDevice* __restrict__ cd,
-                   const DeviceInfo* __restrict__ info, float* __restrict__ u, int64_t d_packed) {
+                   const DeviceInfo* __restrict__ info, float* __restrict__ u, int64_t d_packed, float* __restrict__ w,
+                   float scale) {
     __shared__ double2 bs[kMaxN];
     __shared__ int rows[kMaxN];
     const int count = info->n_active;
@@ -55,8 +56,24 @@ cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const 
                         }
                     }
             }
-            __stcs(reinterpret_cast<float2*>(u + v * 2), make_float2((float)a0, (float)a1));
-            if (PACKED) __stcs(reinterpret_cast<float2*>(u + len + v * 2), make_float2((float)i0, (float)i1));
+            if (u != nullptr) {
+                __stcs(reinterpret_cast<float2*>(u + v * 2), make_float2((float)a0, (float)a1));
+                if (PACKED) __stcs(reinterpret_cast<float2*>(u + len + v * 2), make_float2((float)i0, (float)i1));
+            }
+            if (w != nullptr) {                          // w <- w - scale * u, u rounded to fp32 first as when stored
+                float2* wp = reinterpret_cast<float2*>(w + v * 2);
+                float2 wv = *wp;
+                wv.x = fmaf(-scale, (float)a0, wv.x);
+                wv.y = fmaf(-scale, (float)a1, wv.y);
+                *wp = wv;
+                if (PACKED) {
+                    wp = reinterpret_cast<float2*>(w + len + v * 2);
+                    wv = *wp;
+                    wv.x = fmaf(-scale, (float)i0, wv.x);
+                    wv.y = fmaf(-scale, (float)i1, wv.y);
+                    *wp = wv;
+                }
+            }
         }
     } else {
         for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < len; i += stride) {
@@ -71,8 +88,14 @@ cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const 
                     i0 = fma(b.y, (double)x.x, i0);
                 }
             }
-            u[i] = (float)a0;
-            if (PACKED && len + i < d_packed) u[len + i] = (float)i0;
+            if (u != nullptr) {
+                u[i] = (float)a0;
+                if (PACKED && len + i < d_packed) u[len + i] = (float)i0;
+            }
+            if (w != nullptr) {
+                w[i] = fmaf(-scale, (float)a0, w[i]);
+                if (PACKED && len + i < d_packed) w[len + i] = fmaf(-scale, (float)i0, w[len + i]);
+            }
         }
     }
 }
@@ -80,7 +103,7 @@ cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const 
 }  // namespace
 
 int launch_cyc_recover(draco_plan* p, const float2* R, int64_t len, int64_t ld, float* u, int64_t d_packed,
-                       cudaStream_t st) {
+                       cudaStream_t st, float* w, float scale) {
     const bool packed = d_packed > 0;
     // 64-bit stores of u need len even; in packed mode the second half starts at u + len and must cover it fully
     const bool vec2 = (len % 2 == 0) && (ld % 2 == 0) && (!packed || d_packed == 2 * len);
@@ -90,7 +113,7 @@ int launch_cyc_recover(draco_plan* p, const float2* R, int64_t len, int64_t ld, 
     if (want > cap) want = cap;
     if (want < 1) want = 1;
 #define DRACO_REC(V2, PK) \
-    cyc_recover_kernel<V2, PK><<<(int)want, kThreads, 0, st>>>(R, len, ld, p->cyc_dev, p->info_dev, u, d_packed)
+    cyc_recover_kernel<V2, PK><<<(int)want, kThreads, 0, st>>>(R, len, ld, p->cyc_dev, p->info_dev, u, d_packed, w, scale)
     if (vec2) {
         if (packed) DRACO_REC(true, true); else DRACO_REC(true, false);
     } else {

@@ -258,6 +258,18 @@ int draco_decode(draco_plan* plan, const void* R, const uint8_t* flags, float* u
     return launch_cyc_recover(plan, (const float2*)R, vec_len(plan), vec_len(plan), u, is_packed(plan) ? plan->d : 0, st);
 }
 
+int draco_decode_update(draco_plan* plan, const void* R, const uint8_t* flags, float* w, float scale, void* stream) {
+    if (!plan || !R || !w || !aligned16(R) || !aligned16(w)) return DRACO_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (plan->code == DRACO_REP)
+        return launch_rep_vote(plan, (const float*)R, plan->d, plan->d, nullptr, nullptr, nullptr, true, st, w, scale);
+    if (!flags) return DRACO_EINVAL;
+    int rc = launch_cyc_decode_vector(plan, flags, st);
+    if (rc != DRACO_OK) return rc;
+    return launch_cyc_recover(plan, (const float2*)R, vec_len(plan), vec_len(plan), nullptr, is_packed(plan) ? plan->d : 0, st, w,
+                              scale);
+}
+
 int draco_locate_decode(draco_plan* plan, const void* R, const float* f, uint8_t* flags, float* u, void* stream) {
     if (!plan || !R || !u || !flags || !aligned16(R) || !aligned16(u)) return DRACO_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;

@@ -108,7 +108,7 @@ int cuda_fail(cudaError_t err, const char* what);
 int launch_rep_encode(const draco_plan* p, const float* G, float* Z, int64_t len, int64_t ldg, int64_t ldz,
                       cudaStream_t st);
 int launch_rep_vote(draco_plan* p, const float* R, int64_t len, int64_t ld, float* u, float* maj, uint8_t* flags,
-                    bool reset, cudaStream_t st);
+                    bool reset, cudaStream_t st, float* w = nullptr, float scale = 0.0f);
 int launch_cyc_encode(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz,
                       int64_t half, int64_t d_real, cudaStream_t st);
 int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t len, int64_t ld, bool accumulate,
@@ -117,7 +117,7 @@ int launch_cyc_project_finish(draco_plan* p, double2* e_out, cudaStream_t st);
 int launch_cyc_solve(draco_plan* p, const double2* e, uint8_t* flags, cudaStream_t st);
 int launch_cyc_decode_vector(draco_plan* p, const uint8_t* flags, cudaStream_t st);
 int launch_cyc_recover(draco_plan* p, const float2* R, int64_t len, int64_t ld, float* u, int64_t d_packed,
-                       cudaStream_t st);
+                       cudaStream_t st, float* w = nullptr, float scale = 0.0f);
 int launch_generate(float* out, int rows, int64_t len, int64_t ld, int64_t i0, int row0, float mean, float std,
                     uint64_t seed, cudaStream_t st);
 int launch_corrupt_row(float* row, int64_t nvals, int64_t v0, int model, float param, uint64_t seed, int node,

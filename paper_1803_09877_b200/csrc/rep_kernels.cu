@@ -49,6 +49,19 @@ __device__ __forceinline__ void store_vals(float* ptr, const float (&x)[2]) {
 }
 __device__ __forceinline__ void store_vals(float* ptr, const float (&x)[1]) { __stcs(ptr, x[0]); }
 
+// w <- w - scale * x on VEC consecutive entries (the SGD step of Section 2 fused into the decoder's epilogue)
+__device__ __forceinline__ void update_vals(float* ptr, const float (&x)[4], float scale) {
+    float4 w = *reinterpret_cast<const float4*>(ptr);
+    w.x = fmaf(-scale, x[0], w.x); w.y = fmaf(-scale, x[1], w.y); w.z = fmaf(-scale, x[2], w.z); w.w = fmaf(-scale, x[3], w.w);
+    *reinterpret_cast<float4*>(ptr) = w;
+}
+__device__ __forceinline__ void update_vals(float* ptr, const float (&x)[2], float scale) {
+    float2 w = *reinterpret_cast<const float2*>(ptr);
+    w.x = fmaf(-scale, x[0], w.x); w.y = fmaf(-scale, x[1], w.y);
+    *reinterpret_cast<float2*>(ptr) = w;
+}
+__device__ __forceinline__ void update_vals(float* ptr, const float (&x)[1], float scale) { ptr[0] = fmaf(-scale, x[0], ptr[0]); }
+
 // ---------------------------------------------------------------- encode
 template <int MMAX, int VEC>
 __global__ void __launch_bounds__(kThreads)
@@ -175,7 +188,7 @@ __device__ __forceinline__ void vote_group(const Pack<VEC> (&val)[MMAX], int m, 
 template <int MMAX, int VEC, int GB, int TPB>
 __global__ void __launch_bounds__(TPB)
 rep_vote_kernel(const uint32_t* __restrict__ R, int64_t len, int64_t ld, GroupTable gt, float* __restrict__ u,
-                float* __restrict__ maj, RepScratch* scratch) {
+                float* __restrict__ maj, RepScratch* scratch, float* __restrict__ w, float scale) {
     __shared__ uint32_t smask[kMaxN][MMAX > 0 ? 1 : 4];   // generic path: up to 128 members = 4 words
     for (int i = threadIdx.x; i < kMaxN * (MMAX > 0 ? 1 : 4); i += TPB) (&smask[0][0])[i] = 0;
     __syncthreads();
@@ -257,6 +270,7 @@ rep_vote_kernel(const uint32_t* __restrict__ R, int64_t len, int64_t ld, GroupTa
             }
         }
         if (u != nullptr) store_vals(u + col, acc);
+        if (w != nullptr) update_vals(w + col, acc, scale);
     }
 
     // block totals -> global scratch (integer OR / add: order-independent, hence deterministic)
@@ -336,7 +350,7 @@ int launch_rep_encode(const draco_plan* p, const float* G, float* Z, int64_t len
 }
 
 int launch_rep_vote(draco_plan* p, const float* R, int64_t len, int64_t ld, float* u, float* maj, uint8_t* flags,
-                    bool reset, cudaStream_t st) {
+                    bool reset, cudaStream_t st, float* w, float scale) {
     const GroupTable& gt = p->groups;
     RepScratch* scratch = reinterpret_cast<RepScratch*>(p->mask_dev);
     if (reset) DRACO_CUDA(cudaMemsetAsync(scratch, 0, sizeof(RepScratch), st));
@@ -345,7 +359,7 @@ int launch_rep_vote(draco_plan* p, const float* R, int64_t len, int64_t ld, floa
     const bool generic = gt.max_size > 16;
 #define DRACO_VOTE(MM, VV, GG, TT)                                                                                 \
     rep_vote_kernel<MM, VV, GG, TT><<<grid_for(len / VV, p->sm_count, 8) * (kThreads / TT), TT, 0, st>>>(Rb, len, ld, gt, u, \
-                                                                                                        maj, scratch)
+                                                                                                        maj, scratch, w, scale)
     if (vec4) {
         if (gt.max_size <= 4) DRACO_VOTE(4, 4, 4, 256);
         else if (gt.max_size <= 8) DRACO_VOTE(8, 4, 2, 256);

@@ -403,3 +403,60 @@ def test_packed_full_size_resnet152_sampled():
     uhat = orc.cyc_recover(Ro, orc.cyc_decode_vector(n, s, want_flags))
     floor = normwise(np.concatenate([uhat.real, uhat.imag]), exact)
     assert normwise(host(u[both]), exact) <= 2.0 * floor + 1e-6
+
+
+@pytest.mark.parametrize("code_name,n,s,d", [("CYC", 15, 2, 40_004), ("CYC_PACKED", 15, 2, 40_008), ("CYC_PACKED", 9, 1, 1001)])
+def test_decode_fused_with_model_update(code_name, n, s, d):
+    """w <- w - scale * D(R) in the recovery kernel's epilogue (the SGD step of Section 2)."""
+    import paper_1803_09877_b200 as dr
+    packed = code_name == "CYC_PACKED"
+    plan = dr.Plan(n, s, d, getattr(dr, code_name))
+    G = di.gradient_rows(61, n, d)
+    R = orc.cyc_encode_packed(G, n, s) if packed else orc.cyc_encode(G, n, s)
+    adv = di.choose_adversaries(62, n, s)
+    di.apply_adversaries(R, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=63)
+    flags = np.zeros(n, dtype=np.uint8)
+    flags[adv] = 1
+    uo = orc.cyc_decode_packed(R, n, s, flags.astype(bool), d) if packed else orc.cyc_decode(R, n, s, flags.astype(bool))
+    w0 = di.gradient_rows(64, 1, d)[0]
+    w = dev(w0)
+    scale = np.float32(0.05 / n)
+    plan.decode_update(dev(R), dev(flags), w, float(scale))
+    torch.cuda.synchronize()
+    assert normwise(host(w), w0.astype(np.float64) - float(scale) * uo) <= 1e-6
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.decode(dev(R), dev(flags), u)
+    step = (w0.astype(np.float64) - np.float64(scale) * host(u).astype(np.float64)).astype(np.float32)
+    np.testing.assert_allclose(host(w), step, rtol=2e-7, atol=1e-12)
+    # refused decode (more than 2 s flags) leaves the model untouched
+    flags[:] = 0
+    flags[: 2 * s + 1] = 1
+    w2 = dev(w0)
+    plan.decode_update(dev(R), dev(flags), w2, float(scale))
+    assert plan.info()["status"] == dr.binding.ETOOMANY
+    np.testing.assert_array_equal(host(w2), w0)
+
+
+def test_largest_supported_n():
+    n, s, d = 128, 2, 4100
+    dr, plan = _plan(n, s, d)
+    W, Wo = plan.cyc_W(), orc.cyc_W(n, s)
+    assert np.abs(W - Wo).max() <= 1e-12 * np.abs(Wo).max()
+    G = di.gradient_rows(5, n, d)
+    Z = torch.empty((n, 2 * d), dtype=torch.float32, device="cuda")
+    plan.encode(dev(G), Z)
+    torch.cuda.synchronize()
+    Zo = orc.cyc_encode(G, n, s, dtype=np.complex128)
+    Zg = host(Z, complex64=True)
+    for j in (0, 1, 64, 127):
+        assert np.abs(Zg[j] - Zo[j]).max() <= 1e-6 * np.abs(Zo[j]).max()
+    R = Zo.astype(np.complex64)
+    adv = di.choose_adversaries(6, n, s)
+    di.apply_adversaries(R, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=7)
+    f = di.projection_vector(8, d)
+    want = orc.cyc_locate(R, f, n, s)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    plan.locate(dev(R), dev(f), flags)
+    torch.cuda.synchronize()
+    assert sorted(np.flatnonzero(want["flags"])) == adv.tolist() and want["margin"] > 10
+    np.testing.assert_array_equal(host(flags).astype(bool), want["flags"])

@@ -167,3 +167,38 @@ def test_full_size_resnet18_config_sampled():
     want = orc.rep_decode(Rs, n, s)
     assert normwise(host(u[idx]), want["u"]) <= 1e-5
     assert normwise(host(u[idx]), Gs.astype(np.float64).sum(axis=0)) <= 1e-5
+
+
+def test_decode_fused_with_model_update():
+    """w <- w - scale * D(R) in the vote kernel's epilogue (the SGD step of Section 2)."""
+    n, s, d = 15, 2, 50_004
+    dr, plan = _plan(n, s, d)
+    G, R, adv = _received(n, s, d, 77, s)
+    want = orc.rep_decode(R, n, s)
+    w0 = di.gradient_rows(78, 1, d)[0]
+    w = dev(w0)
+    scale = np.float32(0.01 / n)
+    plan.decode_update(dev(R), None, w, float(scale))
+    torch.cuda.synchronize()
+    expect = w0.astype(np.float64) - float(scale) * want["u"]
+    assert normwise(host(w), expect) <= 1e-6
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.decode(dev(R), None, u)
+    step = (w0.astype(np.float64) - np.float64(scale) * host(u).astype(np.float64)).astype(np.float32)
+    np.testing.assert_allclose(host(w), step, rtol=2e-7, atol=0)
+
+
+def test_largest_supported_n():
+    n, s, d = 128, 3, 2052                                   # 18 groups of 8 / 7
+    dr, plan = _plan(n, s, d)
+    G, R, adv = _received(n, s, d, 99, s)
+    want = orc.rep_decode(R, n, s)
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    plan.locate_decode(dev(R), None, flags, u)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(host(flags).astype(bool), want["flags"])
+    assert normwise(host(u), want["u"]) <= 1e-5
+    import ctypes
+    h = ctypes.c_void_p()
+    assert dr.binding.lib.draco_plan_create(129, 1, 10, dr.REP, ctypes.byref(h)) == dr.binding.EINVAL
