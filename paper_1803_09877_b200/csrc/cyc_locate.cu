@@ -104,6 +104,81 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
     }
 }
 
+// The same projection for many rows per warp (n > 64): the per-lane running sums live in shared
+// memory instead of registers (2 doubles per row and lane would cost 4 * ceil(n / 8) registers and
+// halve the blocks per SM).  Dynamic shared memory: f tile, then sums[ceil(n / 8)][256] double2.
+template <bool VEC2>
+__global__ void __launch_bounds__(kThreads)
+cyc_project_manyrows_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
+                            double2* __restrict__ partial, int accumulate) {
+    extern __shared__ __align__(16) unsigned char proj_smem[];
+    float* fs = reinterpret_cast<float*>(proj_smem);
+    double2* sums = reinterpret_cast<double2*>(proj_smem + sizeof(float) * kProjectTile);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rpw = (n + kProjectWarps - 1) / kProjectWarps;
+    for (int r = 0; r < rpw; ++r) sums[r * kThreads + threadIdx.x] = make_double2(0.0, 0.0);
+
+    const int64_t ntiles = (len + kProjectTile - 1) / kProjectTile;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int64_t c0 = tile * kProjectTile;
+        const int cnt = (int)((len - c0) < kProjectTile ? (len - c0) : kProjectTile);
+        for (int i = threadIdx.x; i < kProjectTile; i += kThreads) fs[i] = (i < cnt) ? __ldcs(f + c0 + i) : 0.0f;
+        __syncthreads();
+        for (int r = 0; r < rpw; ++r) {
+            const int j = warp + r * kProjectWarps;
+            if (j < n) {
+                const float2* row = R + (int64_t)j * ld + c0;
+                double ar = 0.0, ai = 0.0;
+                if (VEC2 && cnt == kProjectTile) {
+                    const float4* row4 = reinterpret_cast<const float4*>(row);
+#pragma unroll 1
+                    for (int step0 = 0; step0 < kProjectTile / 64; step0 += 8) {
+                        float4 v[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) v[q] = __ldcs(row4 + (step0 + q) * 32 + lane);
+                        float pr = 0.f, pi = 0.f;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const float2 ff = *reinterpret_cast<const float2*>(&fs[((step0 + q) * 32 + lane) * 2]);
+                            pr = fmaf(ff.x, v[q].x, pr); pi = fmaf(ff.x, v[q].y, pi);
+                            pr = fmaf(ff.y, v[q].z, pr); pi = fmaf(ff.y, v[q].w, pi);
+                        }
+                        ar += (double)pr;
+                        ai += (double)pi;
+                    }
+                } else {
+                    for (int i = lane; i < cnt; i += 32) {
+                        const float2 v = __ldcs(row + i);
+                        const float ff = fs[i];
+                        ar += (double)(ff * v.x);
+                        ai += (double)(ff * v.y);
+                    }
+                }
+                double2 s = sums[r * kThreads + threadIdx.x];      // this thread's own slot: no synchronisation needed
+                s.x += ar;
+                s.y += ai;
+                sums[r * kThreads + threadIdx.x] = s;
+            }
+        }
+        __syncthreads();
+    }
+    for (int r = 0; r < rpw; ++r) {
+        const double2 s = sums[r * kThreads + threadIdx.x];
+        double a = s.x, b = s.y;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, off);
+            b += __shfl_xor_sync(0xffffffffu, b, off);
+        }
+        const int j = warp + r * kProjectWarps;
+        if (lane == 0 && j < n) {
+            double2* dst = partial + (int64_t)blockIdx.x * n + j;
+            if (accumulate) { a += dst->x; b += dst->y; }
+            *dst = make_double2(a, b);
+        }
+    }
+}
+
 // e_j = sum over blocks, fixed order.
 __global__ void cyc_project_finish_kernel(const double2* __restrict__ partial, int grid, int n, double2* e) {
     const int j = threadIdx.x;
@@ -299,13 +374,24 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ partial, int grid, c
         if (e_in != nullptr) {
             v = e_in[tid];
         } else {
-            double a = 0.0, b = 0.0;
-            for (int blk = 0; blk < grid; ++blk) {
-                const double2 p = partial[(int64_t)blk * n + tid];
-                a += p.x;
-                b += p.y;
+            // four interleaved running sums (blocks 0,4,8.. / 1,5,9.. / ..) keep the loads independent;
+            // the order is fixed, so the result is still reproducible bit for bit
+            double a[4] = {0.0, 0.0, 0.0, 0.0}, b[4] = {0.0, 0.0, 0.0, 0.0};
+            int blk = 0;
+            for (; blk + 4 <= grid; blk += 4) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const double2 p = partial[(int64_t)(blk + q) * n + tid];
+                    a[q] += p.x;
+                    b[q] += p.y;
+                }
             }
-            v = make_double2(a, b);
+            for (; blk < grid; ++blk) {
+                const double2 p = partial[(int64_t)blk * n + tid];
+                a[0] += p.x;
+                b[0] += p.y;
+            }
+            v = make_double2((a[0] + a[1]) + (a[2] + a[3]), (b[0] + b[1]) + (b[2] + b[3]));
         }
         e[tid] = v;
         cd->e[tid] = v;
@@ -504,6 +590,9 @@ cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n
 
 }  // namespace
 
+// Blocks of the projection: four per SM (six measured slower at n = 15); three per SM is what the
+// shared-memory sums of the n > 64 kernel allow.
+int project_grid_size(int sm_count, int n) { return sm_count * (n <= 64 ? 4 : 3); }
 int project_grid_size(int sm_count) { return sm_count * 4; }
 
 int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t len, int64_t ld, bool accumulate,
@@ -513,14 +602,25 @@ int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t l
     const int n = p->n;
 #define DRACO_PROJ(RPW, V2) \
     cyc_project_kernel<RPW, V2><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0)
-    if (vec2) {
+    if (n > 64) {
+        const size_t smem = sizeof(float) * kProjectTile + sizeof(double2) * kThreads * ((n + kProjectWarps - 1) / kProjectWarps);
+        static bool configured_dev[64] = {};
+        bool& configured = configured_dev[(p->device >= 0 && p->device < 64) ? p->device : 0];
+        if (!configured) {
+            DRACO_CUDA(cudaFuncSetAttribute(cyc_project_manyrows_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)(sizeof(float) * kProjectTile + sizeof(double2) * kThreads * 16)));
+            DRACO_CUDA(cudaFuncSetAttribute(cyc_project_manyrows_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)(sizeof(float) * kProjectTile + sizeof(double2) * kThreads * 16)));
+            configured = true;
+        }
+        if (vec2) cyc_project_manyrows_kernel<true><<<grid, kThreads, smem, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
+        else cyc_project_manyrows_kernel<false><<<grid, kThreads, smem, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
+    } else if (vec2) {
         if (n <= 32) DRACO_PROJ(4, true);
-        else if (n <= 64) DRACO_PROJ(8, true);
-        else DRACO_PROJ(16, true);
+        else DRACO_PROJ(8, true);
     } else {
         if (n <= 32) DRACO_PROJ(4, false);
-        else if (n <= 64) DRACO_PROJ(8, false);
-        else DRACO_PROJ(16, false);
+        else DRACO_PROJ(8, false);
     }
 #undef DRACO_PROJ
     DRACO_CUDA(cudaGetLastError());

@@ -169,7 +169,7 @@ int draco_plan_create(int n, int s, int64_t d, int code, draco_plan** out) {
         DRACO_TRY(cudaMalloc(&p->taps_full_dev, sizeof(float2) * taps_full.size()));
         DRACO_TRY(cudaMemcpy(p->taps_full_dev, taps_full.data(), sizeof(float2) * taps_full.size(),
                              cudaMemcpyHostToDevice));
-        p->project_grid = project_grid_size(p->sm_count);
+        p->project_grid = project_grid_size(p->sm_count, n);
         DRACO_TRY(cudaMalloc(&p->partial_dev, sizeof(double2) * (size_t)p->project_grid * n));
         DRACO_TRY(cudaMemset(p->partial_dev, 0, sizeof(double2) * (size_t)p->project_grid * n));
     }

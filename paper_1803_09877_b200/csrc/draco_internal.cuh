@@ -123,5 +123,6 @@ int launch_generate(float* out, int rows, int64_t len, int64_t ld, int64_t i0, i
 int launch_corrupt_row(float* row, int64_t nvals, int64_t v0, int model, float param, uint64_t seed, int node,
                        bool is_complex, cudaStream_t st);
 int project_grid_size(int sm_count);
+int project_grid_size(int sm_count, int n);
 
 }  // namespace draco

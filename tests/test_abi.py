@@ -43,3 +43,14 @@ def test_argument_checks_need_no_device():
     assert binding.lib.draco_plan_create(15, 2, 10, 7, ctypes.byref(h)) == binding.EINVAL
     assert binding.lib.draco_plan_create(200, 2, 10, binding.CYC, ctypes.byref(h)) == binding.EINVAL
     assert binding.lib.draco_encode(None, None, None, None) == binding.EINVAL
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    """There is no CPU fallback: without libdraco.so the binding refuses to load."""
+    import pytest
+    from paper_1803_09877_b200 import build
+    build.build()
+    from paper_1803_09877_b200 import binding
+    monkeypatch.setattr(binding, "_PKG", "/nonexistent-directory")
+    with pytest.raises(binding.DracoError, match="no CPU fallback"):
+        binding._load()

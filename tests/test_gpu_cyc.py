@@ -460,3 +460,19 @@ def test_largest_supported_n():
     torch.cuda.synchronize()
     assert sorted(np.flatnonzero(want["flags"])) == adv.tolist() and want["margin"] > 10
     np.testing.assert_array_equal(host(flags).astype(bool), want["flags"])
+
+
+def test_rank_cutoff_theta_is_adjustable():
+    """With an absurdly high cutoff every singular value counts as zero: nobody is flagged."""
+    n, s, d = 15, 2, 8192
+    dr, plan = _plan(n, s, d)
+    G, R, adv, f = _received(n, s, d, 321, s)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    plan.locate(dev(R), dev(f), flags)
+    assert sorted(np.flatnonzero(host(flags))) == adv.tolist()
+    plan.set_theta(1e9)
+    plan.locate(dev(R), dev(f), flags)
+    info = plan.info()
+    assert info["locator_rank"] == 0 and info["n_flagged"] == 0 and not host(flags).any()
+    want = orc.cyc_locate(R, f, n, s, theta=1e9)
+    assert want["rank"] == 0 and not want["flags"].any()
