@@ -19,7 +19,7 @@ namespace draco {
 namespace {
 
 constexpr int kThreads = kProjectWarps * 32;
-constexpr int kSolveThreads = 128;
+constexpr int kSolveThreads = 512;
 
 __device__ __forceinline__ double2 cmul(double2 a, double2 b) {
     return make_double2(a.x * b.x - a.y * b.y, a.x * b.y + a.y * b.x);
@@ -104,6 +104,98 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
     }
 }
 
+// The same projection for few rows (n <= 16): with one or two rows per warp the block-wide tile
+// barriers of the kernel above dominate, so here every warp works alone on 256-coordinate chunks
+// of all n rows, with f for its chunk in registers (8 values per lane) and no shared memory or
+// barrier in the loop.  Per-lane running sums in fp64 registers (2 n doubles).
+template <bool VEC2>
+__global__ void __launch_bounds__(kThreads)
+cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
+                           double2* __restrict__ partial, int accumulate) {
+    constexpr int NMAX = 16, CH = 256;
+    __shared__ double2 wsum[kProjectWarps][NMAX];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    double accr[NMAX], acci[NMAX];
+#pragma unroll
+    for (int j = 0; j < NMAX; ++j) { accr[j] = 0.0; acci[j] = 0.0; }
+    const int64_t nchunks = (len + CH - 1) / CH;
+    const int64_t nwarps = (int64_t)gridDim.x * kProjectWarps;
+    for (int64_t chunk = (int64_t)blockIdx.x * kProjectWarps + warp; chunk < nchunks; chunk += nwarps) {
+        const int64_t c0 = chunk * CH;
+        const int cnt = (int)((len - c0) < CH ? (len - c0) : CH);
+        if (VEC2 && cnt == CH) {
+            float2 ff[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) ff[q] = __ldcs(reinterpret_cast<const float2*>(f + c0) + q * 32 + lane);
+#pragma unroll
+            for (int jj = 0; jj < NMAX; jj += 2) {
+                if (jj < n) {
+                    float4 va[4], vb[4];
+                    const float4* ra = reinterpret_cast<const float4*>(R + (int64_t)jj * ld + c0);
+                    const bool two = jj + 1 < n;
+                    const float4* rb = reinterpret_cast<const float4*>(R + (int64_t)(two ? jj + 1 : jj) * ld + c0);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) va[q] = __ldcs(ra + q * 32 + lane);
+                    if (two) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) vb[q] = __ldcs(rb + q * 32 + lane);
+                    }
+                    float pr = 0.f, pi = 0.f;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        pr = fmaf(ff[q].x, va[q].x, pr); pi = fmaf(ff[q].x, va[q].y, pi);
+                        pr = fmaf(ff[q].y, va[q].z, pr); pi = fmaf(ff[q].y, va[q].w, pi);
+                    }
+                    accr[jj] += (double)pr;
+                    acci[jj] += (double)pi;
+                    if (two) {
+                        pr = 0.f; pi = 0.f;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            pr = fmaf(ff[q].x, vb[q].x, pr); pi = fmaf(ff[q].x, vb[q].y, pi);
+                            pr = fmaf(ff[q].y, vb[q].z, pr); pi = fmaf(ff[q].y, vb[q].w, pi);
+                        }
+                        accr[jj + 1] += (double)pr;
+                        acci[jj + 1] += (double)pi;
+                    }
+                }
+            }
+        } else {
+            for (int i = lane; i < cnt; i += 32) {
+                const float fi = __ldcs(f + c0 + i);
+#pragma unroll
+                for (int j = 0; j < NMAX; ++j)
+                    if (j < n) {
+                        const float2 v = __ldcs(R + (int64_t)j * ld + c0 + i);
+                        accr[j] += (double)(fi * v.x);
+                        acci[j] += (double)(fi * v.y);
+                    }
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < NMAX; ++j) {
+        double a = accr[j], b = acci[j];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, off);
+            b += __shfl_xor_sync(0xffffffffu, b, off);
+        }
+        if (lane == 0) wsum[warp][j] = make_double2(a, b);
+    }
+    __syncthreads();
+    if (threadIdx.x < n) {
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < kProjectWarps; ++w) {            // fixed order: reproducible
+            a += wsum[w][threadIdx.x].x;
+            b += wsum[w][threadIdx.x].y;
+        }
+        double2* dst = partial + (int64_t)blockIdx.x * n + threadIdx.x;
+        if (accumulate) { a += dst->x; b += dst->y; }
+        *dst = make_double2(a, b);
+    }
+}
+
 // The same projection for many rows per warp (n > 64): the per-lane running sums live in shared
 // memory instead of registers (2 doubles per row and lane would cost 4 * ceil(n / 8) registers and
 // halve the blocks per SM).  Dynamic shared memory: f tile, then sums[ceil(n / 8)][256] double2.
@@ -179,17 +271,29 @@ cyc_project_manyrows_kernel(const float2* __restrict__ R, const float* __restric
     }
 }
 
-// e_j = sum over blocks, fixed order.
-__global__ void cyc_project_finish_kernel(const double2* __restrict__ partial, int grid, int n, double2* e) {
-    const int j = threadIdx.x;
-    if (j < n) {
-        double a = 0.0, b = 0.0;
-        for (int blk = 0; blk < grid; ++blk) {
-            const double2 p = partial[(int64_t)blk * n + j];
-            a += p.x;
-            b += p.y;
-        }
-        e[j] = make_double2(a, b);
+// e_j = sum over the blocks' partials: one warp per row, lane l takes blocks l, l+32, .., then a
+// butterfly over the lanes.  The order is fixed, so the sum is reproducible bit for bit.
+__device__ __forceinline__ double2 sum_partials_row(const double2* __restrict__ partial, int grid, int n, int j, int lane) {
+    double a = 0.0, b = 0.0;
+    for (int blk = lane; blk < grid; blk += 32) {
+        const double2 p = partial[(int64_t)blk * n + j];
+        a += p.x;
+        b += p.y;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, off);
+        b += __shfl_xor_sync(0xffffffffu, b, off);
+    }
+    return make_double2(a, b);
+}
+
+__global__ void __launch_bounds__(1024)
+cyc_project_finish_kernel(const double2* __restrict__ partial, int grid, int n, double2* e) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (int j = warp; j < n; j += nwarps) {
+        const double2 v = sum_partials_row(partial, grid, n, j, lane);
+        if (lane == 0) e[j] = v;
     }
 }
 
@@ -369,31 +473,18 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ partial, int grid, c
     const int tid = threadIdx.x;
     const double rsn = 1.0 / sqrt((double)n);
 
-    if (tid < n) {
-        double2 v;
-        if (e_in != nullptr) {
-            v = e_in[tid];
-        } else {
-            // four interleaved running sums (blocks 0,4,8.. / 1,5,9.. / ..) keep the loads independent;
-            // the order is fixed, so the result is still reproducible bit for bit
-            double a[4] = {0.0, 0.0, 0.0, 0.0}, b[4] = {0.0, 0.0, 0.0, 0.0};
-            int blk = 0;
-            for (; blk + 4 <= grid; blk += 4) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const double2 p = partial[(int64_t)(blk + q) * n + tid];
-                    a[q] += p.x;
-                    b[q] += p.y;
-                }
-            }
-            for (; blk < grid; ++blk) {
-                const double2 p = partial[(int64_t)blk * n + tid];
-                a[0] += p.x;
-                b[0] += p.y;
-            }
-            v = make_double2((a[0] + a[1]) + (a[2] + a[3]), (b[0] + b[1]) + (b[2] + b[3]));
+    if (e_in == nullptr) {
+        const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
+        for (int j = warp; j < n; j += nwarps) {
+            const double2 v = sum_partials_row(partial, grid, n, j, lane);
+            if (lane == 0) e[j] = v;
         }
-        e[tid] = v;
+    } else if (tid < n) {
+        e[tid] = e_in[tid];
+    }
+    __syncthreads();
+    if (tid < n) {
+        const double2 v = e[tid];
         cd->e[tid] = v;
         mag[tid] = sqrt(cabs2(v));
         h[tid] = make_double2(0.0, 0.0);
@@ -615,6 +706,9 @@ int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t l
         }
         if (vec2) cyc_project_manyrows_kernel<true><<<grid, kThreads, smem, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
         else cyc_project_manyrows_kernel<false><<<grid, kThreads, smem, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
+    } else if (n <= 16) {
+        if (vec2) cyc_project_fewrows_kernel<true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
+        else cyc_project_fewrows_kernel<false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
     } else if (vec2) {
         if (n <= 32) DRACO_PROJ(4, true);
         else DRACO_PROJ(8, true);
@@ -628,7 +722,7 @@ int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t l
 }
 
 int launch_cyc_project_finish(draco_plan* p, double2* e_out, cudaStream_t st) {
-    cyc_project_finish_kernel<<<1, kMaxN, 0, st>>>(p->partial_dev, p->project_grid, p->n, e_out);
+    cyc_project_finish_kernel<<<1, 1024, 0, st>>>(p->partial_dev, p->project_grid, p->n, e_out);
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }
@@ -710,7 +804,7 @@ extern "C" int draco_cyc_project_noalloc(int n, int64_t d, const void* R, const 
         else cyc_project_kernel<16, false><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
     }
     DRACO_CUDA(cudaGetLastError());
-    cyc_project_finish_kernel<<<1, kMaxN, 0, st>>>(partial, grid, n, reinterpret_cast<double2*>(e));
+    cyc_project_finish_kernel<<<1, 1024, 0, st>>>(partial, grid, n, reinterpret_cast<double2*>(e));
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }
