@@ -108,7 +108,7 @@ struct RingState {
 // MODE 2: anything (run-time guards).  Returns false when a wait gave up.
 template <int S, int P, int MODE, bool PACKED>
 __device__ __forceinline__ bool encode_step(Window<S>& w, RingState& rs, int vv, int n, const float* ring_t,
-                                            float* stash_t, float2* zcol, int64_t ldz, bool active, int lane,
+                                            float* stash_t, float2* zcol, int64_t ldz, int active, int lane,
                                             const EncodeTaps& taps, const EncodeTaps64& taps64,
                                             const EncodePhase64& ph64) {
     constexpr int R = Window<S>::R, NBIG = Window<S>::NBIG, H = Window<S>::H, SL = Window<S>::SL;
@@ -129,8 +129,10 @@ __device__ __forceinline__ bool encode_step(Window<S>& w, RingState& rs, int vv,
             const float2 a = *reinterpret_cast<const float2*>(ring_t + rs.st * kTile);
             const float2 b = *reinterpret_cast<const float2*>(ring_t + rs.st * kTile + kTile / 2);
             x = make_float4(a.x, a.y, b.x, b.y);
-        } else {
-            x = *reinterpret_cast<const float4*>(ring_t + rs.st * kTile);
+        } else {           // coordinates 2l, 2l+1 and 64+2l, 64+2l+1 of the warp's 128: see the stores below
+            const float2 a = *reinterpret_cast<const float2*>(ring_t + rs.st * kTile);
+            const float2 b = *reinterpret_cast<const float2*>(ring_t + rs.st * kTile + 64);
+            x = make_float4(a.x, a.y, b.x, b.y);
         }
         rs.pend_bar = rs.empty0 + 8 * rs.st;
         rs.pend_bits = __float_as_uint(x.x);
@@ -189,15 +191,18 @@ __device__ __forceinline__ bool encode_step(Window<S>& w, RingState& rs, int vv,
         }
         if (PACKED) {
             // components 0,1 filtered the real parts (X), 2,3 the imaginary parts (Y): z = X + i Y
-            if (active) {
+            if (active & 1) {
                 float4* dst = reinterpret_cast<float4*>(zcol + (int64_t)j * ldz);
                 __stcs(dst, make_float4((float)(xr[0] - xi[2]), (float)(xi[0] + xr[2]), (float)(xr[1] - xi[3]),
                                         (float)(xi[1] + xr[3])));
             }
-        } else if (active) {
-            float4* dst = reinterpret_cast<float4*>(zcol + (int64_t)j * ldz);
-            __stcs(dst, make_float4((float)xr[0], (float)xi[0], (float)xr[1], (float)xi[1]));
-            __stcs(dst + 1, make_float4((float)xr[2], (float)xi[2], (float)xr[3], (float)xi[3]));
+        } else {
+            // A lane's two 16-byte stores are 512 bytes apart, so that each store instruction of the warp
+            // covers 512 contiguous bytes (whole 32-byte sectors).  With the 4 coordinates of a lane adjacent,
+            // every instruction wrote half of 32 sectors and the kernel stopped at 4.9 TB/s.
+            float2* dst = zcol + (int64_t)j * ldz;
+            if (active & 1) __stcs(reinterpret_cast<float4*>(dst), make_float4((float)xr[0], (float)xi[0], (float)xr[1], (float)xi[1]));
+            if (active & 2) __stcs(reinterpret_cast<float4*>(dst + 64), make_float4((float)xr[2], (float)xi[2], (float)xr[3], (float)xi[3]));
         }
     }
     return true;
@@ -205,7 +210,7 @@ __device__ __forceinline__ bool encode_step(Window<S>& w, RingState& rs, int vv,
 
 template <int S, int MODE, bool PACKED, int P = 0>
 __device__ __forceinline__ bool encode_chunk(Window<S>& w, RingState& rs, int v0, int n, const float* ring_t,
-                                             float* stash_t, float2* zcol, int64_t ldz, bool active, int lane,
+                                             float* stash_t, float2* zcol, int64_t ldz, int active, int lane,
                                              const EncodeTaps& taps, const EncodeTaps64& taps64,
                                              const EncodePhase64& ph64) {
     if constexpr (P < Window<S>::SL) {
@@ -280,13 +285,15 @@ cyc_encode_ring_kernel(const float* __restrict__ G, float2* __restrict__ Z, int6
     RingState rs;
     rs.full0 = full0; rs.empty0 = empty0; rs.st = 0; rs.par = 0;
     rs.pend_bar = 0; rs.pend_bits = 0; rs.pending = false;
-    const float* ring_t = ring + tid * kPerThread;
+    // unpacked: a lane owns coordinates 2l, 2l+1, 64+2l, 64+2l+1 of its warp's 128; packed: entries 2 tid, 2 tid + 1
+    const int first = PACKED ? tid * 2 : warp * 128 + lane * 2;
+    const float* ring_t = ring + first;
     float* stash_t = stash + tid * kVec;
     const int total = n + 2 * S;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const int64_t c0 = tile * kTileCoords;
-        const bool active = c0 + tid * kPerThread < len;
-        float2* zcol = Z + c0 + tid * kPerThread;
+        const int active = (c0 + first < len ? 1 : 0) | ((PACKED || c0 + first + 64 < len) ? 2 : 0);
+        float2* zcol = Z + c0 + first;
         bool ok = true;
         int v0 = 0;
         if (n >= SL && S > 0) {
