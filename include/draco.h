@@ -188,7 +188,10 @@ int draco_get_info(draco_plan* plan, draco_info* info /*host*/, void* stream);
 /*
  * Whole path with host buffers (pageable or pinned): copies G and f to the device in
  * column chunks, encodes, applies the given adversaries, locates, decodes, and copies
- * u and flags back.  Synchronous.  Z (device [n][d], caller-owned) keeps the received matrix.
+ * u and flags back.  Synchronous: waits for the device's earlier work on entry, runs on two internal streams (the copy
+ * of one chunk overlaps the kernels of the previous one) and returns when u and flags are on the host.  The first call
+ * on a plan allocates two staging buffers (n x 2 x chunk floats), u and f on the device.
+ * Z (device, one row per node, caller-owned) keeps the received matrix.
  */
 int draco_pipeline_host(draco_plan* plan, const float* G_host, const float* f_host,
                         const int* adv_idx /*host*/, const int* adv_model /*host*/, const float* adv_param /*host*/,

@@ -116,6 +116,12 @@ void free_plan(draco_plan* p) {
     if (p->flags_dev) cudaFree(p->flags_dev);
     if (p->mask_dev) cudaFree(p->mask_dev);
     if (p->stage_dev) cudaFree(p->stage_dev);
+    if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
+    if (p->work_stream) cudaStreamDestroy(p->work_stream);
+    for (int b = 0; b < 2; ++b) {
+        if (p->ev_copied[b]) cudaEventDestroy(p->ev_copied[b]);
+        if (p->ev_consumed[b]) cudaEventDestroy(p->ev_consumed[b]);
+    }
     if (p->f_dev) cudaFree(p->f_dev);
     if (p->u_dev) cudaFree(p->u_dev);
     delete p;
@@ -347,43 +353,59 @@ int draco_pipeline_host(draco_plan* plan, const float* G_host, const float* f_ho
     int64_t chunk = ((int64_t)64 << 20) / n;
     chunk = (chunk / (2 * kProjectTile)) * (2 * kProjectTile);
     if (chunk < 2 * kProjectTile) chunk = 2 * kProjectTile;
-    if (!plan->stage_dev) {
-        DRACO_CUDA(cudaMalloc(&plan->stage_dev, sizeof(float) * (size_t)n * chunk));
+    if (!plan->stage_dev) {                            // two staging buffers: the copy of chunk i+1 overlaps the kernels of chunk i
+        DRACO_CUDA(cudaMalloc(&plan->stage_dev, sizeof(float) * (size_t)n * chunk * 2));
         plan->stage_chunk = chunk;
+        DRACO_CUDA(cudaStreamCreateWithFlags(&plan->copy_stream, cudaStreamNonBlocking));
+        DRACO_CUDA(cudaStreamCreateWithFlags(&plan->work_stream, cudaStreamNonBlocking));
+        for (int b = 0; b < 2; ++b) {
+            DRACO_CUDA(cudaEventCreateWithFlags(&plan->ev_copied[b], cudaEventDisableTiming));
+            DRACO_CUDA(cudaEventCreateWithFlags(&plan->ev_consumed[b], cudaEventDisableTiming));
+        }
     }
     if (!plan->u_dev) DRACO_CUDA(cudaMalloc(&plan->u_dev, sizeof(float) * (size_t)d));
     if (cyc && !plan->f_dev) DRACO_CUDA(cudaMalloc(&plan->f_dev, sizeof(float) * (size_t)vlen));
     chunk = plan->stage_chunk;
     const int64_t step = packed ? chunk / 2 : chunk;   // vector entries per chunk
-    cudaStream_t st = 0;
+    DRACO_CUDA(cudaDeviceSynchronize());               // earlier work of the caller that touches Z or the plan
+    cudaStream_t st = plan->work_stream, cst = plan->copy_stream;
     if (cyc) DRACO_CUDA(cudaMemcpyAsync(plan->f_dev, f_host, sizeof(float) * (size_t)vlen, cudaMemcpyHostToDevice, st));
     bool first = true;
-    for (int64_t c0 = 0; c0 < vlen; c0 += step) {
+    int64_t chunk_no = 0;
+    for (int64_t c0 = 0; c0 < vlen; c0 += step, ++chunk_no) {
         const int64_t len = (vlen - c0) < step ? (vlen - c0) : step;
-        DRACO_CUDA(cudaMemcpy2DAsync(plan->stage_dev, sizeof(float) * (size_t)chunk, G_host + c0, sizeof(float) * (size_t)d,
-                                     sizeof(float) * (size_t)len, n, cudaMemcpyHostToDevice, st));
+        const int buf = (int)(chunk_no & 1);
+        float* stage = plan->stage_dev + (size_t)buf * n * chunk;
+        if (chunk_no >= 2) DRACO_CUDA(cudaStreamWaitEvent(cst, plan->ev_consumed[buf], 0));
+        DRACO_CUDA(cudaMemcpy2DAsync(stage, sizeof(float) * (size_t)chunk, G_host + c0, sizeof(float) * (size_t)d,
+                                     sizeof(float) * (size_t)len, n, cudaMemcpyHostToDevice, cst));
         int rc;
         if (cyc) {
             int64_t half = 0, d_stage = len;
             if (packed) {                              // second half of the gradient next to the first in the stage
                 const int64_t len_b = (d - vlen - c0) < len ? (d - vlen - c0) : len;
                 if (len_b > 0)
-                    DRACO_CUDA(cudaMemcpy2DAsync(plan->stage_dev + step, sizeof(float) * (size_t)chunk, G_host + vlen + c0,
+                    DRACO_CUDA(cudaMemcpy2DAsync(stage + step, sizeof(float) * (size_t)chunk, G_host + vlen + c0,
                                                  sizeof(float) * (size_t)d, sizeof(float) * (size_t)len_b, n,
-                                                 cudaMemcpyHostToDevice, st));
+                                                 cudaMemcpyHostToDevice, cst));
                 half = step;
                 d_stage = step + (len_b > 0 ? len_b : 0);
             }
+            DRACO_CUDA(cudaEventRecord(plan->ev_copied[buf], cst));
+            DRACO_CUDA(cudaStreamWaitEvent(st, plan->ev_copied[buf], 0));
             float2* Zc = (float2*)Z + c0;
-            rc = launch_cyc_encode(plan, plan->stage_dev, Zc, len, chunk, vlen, half, d_stage, st);
+            rc = launch_cyc_encode(plan, stage, Zc, len, chunk, vlen, half, d_stage, st);
             if (rc == DRACO_OK) rc = corrupt_range(plan, Z, c0, len, vlen, adv_idx, adv_model, adv_param, n_adv, adv_seed, st);
             if (rc == DRACO_OK) rc = launch_cyc_project(plan, Zc, plan->f_dev + c0, len, vlen, !first, st);
         } else {
+            DRACO_CUDA(cudaEventRecord(plan->ev_copied[buf], cst));
+            DRACO_CUDA(cudaStreamWaitEvent(st, plan->ev_copied[buf], 0));
             float* Zc = (float*)Z + c0;
-            rc = launch_rep_encode(plan, plan->stage_dev, Zc, len, chunk, d, st);
+            rc = launch_rep_encode(plan, stage, Zc, len, chunk, d, st);
             if (rc == DRACO_OK) rc = corrupt_range(plan, Z, c0, len, d, adv_idx, adv_model, adv_param, n_adv, adv_seed, st);
         }
         if (rc != DRACO_OK) return rc;
+        DRACO_CUDA(cudaEventRecord(plan->ev_consumed[buf], st));
         first = false;
     }
     int rc;

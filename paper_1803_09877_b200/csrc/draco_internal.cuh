@@ -87,7 +87,9 @@ struct draco_plan {
     uint8_t* flags_dev;               // [n] internal flags
     uint32_t* mask_dev;               // repetition: disagreement bits, [n] words
     // host-buffer pipeline (allocated on its first call)
-    float* stage_dev;                 // [n][stage_chunk] slice of G
+    float* stage_dev;                 // two [n][stage_chunk] slices of G (double buffer)
+    cudaStream_t copy_stream, work_stream;
+    cudaEvent_t ev_copied[2], ev_consumed[2];
     int64_t stage_chunk;
     float* f_dev;                     // [d]
     float* u_dev;                     // [d]
