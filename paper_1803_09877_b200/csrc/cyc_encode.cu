@@ -11,10 +11,10 @@
 // rotation per output.  The taps do not depend on j, so they sit in the kernel's constant
 // parameter bank and every multiply-add takes its coefficient from there.
 //
-// Data movement.  A thread block owns a tile of 1536 coordinates and walks the n rows once.
-// One producer lane streams the row tiles (6 KB each) from global memory into a ring of
+// Data movement.  A thread block owns a tile of 1536 coordinates (1408 for s >= 6) and walks the n rows
+// once.  One producer lane streams the row tiles (6 KB each) from global memory into a ring of
 // shared-memory stages with bulk asynchronous copies (cp.async.bulk + mbarrier, no
-// multicast); 12 consumer warps take each row from the ring into a register window of the
+// multicast); 12 (11) consumer warps take each row from the ring into a register window of the
 // last 2 s + 1 rows, 4 coordinates per thread.  The first 2 s rows are also kept in shared
 // memory, because the circle closes on them at the end of the walk; nothing is read twice.
 // HBM traffic is the algorithmic minimum: 4 n len bytes read + 8 n len bytes written.
@@ -31,11 +31,18 @@ namespace draco {
 
 namespace {
 
-constexpr int kConsumers = 384;                 // consumer threads (12 warps); the next warp is the producer
-constexpr int kRingThreads = kConsumers + 32;
 constexpr int kVec = 4;                         // coordinates per consumer thread
-constexpr int kTile = kConsumers * kVec;        // coordinates per tile = floats per stage
-constexpr int kStages = 16;                     // ring depth (96 KB in flight per block)
+// Block shape per s.  A scheduler's 16 K registers cap a thread at 128 registers once it hosts 4 warps,
+// and the s >= 6 window needs about 155: those kernels run 11 consumer warps + the producer (3 warps per
+// scheduler) instead of 12 + 1 (measured at n = 45: 7.1 ms against 8.0 ms with spills; for s = 5 the
+// 12-warp shape is the faster one, 6.0 ms against 6.4 ms).
+template <int S>
+struct RingCfg {
+    static constexpr int kConsumers = S >= 6 ? 352 : 384;    // consumer threads; the next warp is the producer
+    static constexpr int kThreads = kConsumers + 32;
+    static constexpr int kTile = kConsumers * kVec;           // coordinates per tile = floats per stage
+};
+constexpr int kStages = 16;                     // ring depth (up to 96 KB in flight per block)
 static_assert((kStages & (kStages - 1)) == 0, "stage indices and parities are derived with masks: kStages must be a power of two");
 constexpr int kGenericThreads = 256;
 
@@ -112,6 +119,7 @@ __device__ __forceinline__ bool encode_step(Window<S>& w, RingState& rs, int vv,
                                             const EncodeTaps& taps, const EncodeTaps64& taps64,
                                             const EncodePhase64& ph64) {
     constexpr int R = Window<S>::R, NBIG = Window<S>::NBIG, H = Window<S>::H, SL = Window<S>::SL;
+    constexpr int kTile = RingCfg<S>::kTile;
     const int total = n + 2 * S;
     if (MODE == 2 && vv >= total) return true;
     const bool from_ring = (MODE != 2) || (vv < n);
@@ -226,13 +234,14 @@ __device__ __forceinline__ bool encode_chunk(Window<S>& w, RingState& rs, int v0
 // coordinates, a tile holds kTile / 2 of them, and a stage receives two slices of each row:
 // G[r][c0 ..] (real parts) and G[r][half + c0 ..] (imaginary parts).
 template <int S, bool PACKED>
-__global__ void __launch_bounds__(kRingThreads)
+__global__ void __launch_bounds__(RingCfg<S>::kThreads, 1)
 cyc_encode_ring_kernel(const float* __restrict__ G, float2* __restrict__ Z, int64_t len, int64_t ldg, int64_t ldz,
                        int64_t half, int n,
                        const __grid_constant__ EncodeTaps taps, const __grid_constant__ EncodeTaps64 taps64,
                        const __grid_constant__ EncodePhase64 ph64, int* err) {
     constexpr int SL = Window<S>::SL;
     constexpr int NSTASH = S > 0 ? 2 * S : 1;
+    constexpr int kConsumers = RingCfg<S>::kConsumers, kTile = RingCfg<S>::kTile;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float* ring = reinterpret_cast<float*>(smem_raw);                        // [kStages][kTile]
     float* stash = ring + kStages * kTile;                                   // [2 S][kTile]
@@ -352,6 +361,7 @@ template <int S, bool PACKED>
 int launch_ring(const draco_plan* p, const float* G, float2* Z, int64_t len, int64_t ldg, int64_t ldz, int64_t half,
                 cudaStream_t st) {
     constexpr int NSTASH = S > 0 ? 2 * S : 1;
+    constexpr int kTile = RingCfg<S>::kTile, kRingThreads = RingCfg<S>::kThreads;
     const size_t smem = sizeof(float) * kTile * (kStages + NSTASH) + 16 * kStages;
     auto kern = cyc_encode_ring_kernel<S, PACKED>;
     static bool configured[64] = {};
