@@ -212,6 +212,7 @@ def run_gpu(args):
     import torch.distributed as dist
 
     import paper_1803_09877_b200 as dr
+    from paper_1803_09877_b200.sharding import locate_sharded, merge_flags
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -252,10 +253,8 @@ def run_gpu(args):
         plan.corrupt(Z, adv, model, param, seed=SEED + 2)
         mark(2)
         if cyc:
-            if world > 1:
-                plan.cyc_project(Z, f, e)
-                dist.all_reduce(e)
-                plan.cyc_locate_from_projection(e, flags)
+            if world > 1:      # d-sharded: local projection, all-reduce of the 2 n doubles, local solve
+                locate_sharded(plan, Z, f, flags, e)
             else:
                 plan.locate(Z, f, flags)
             mark(3)
@@ -263,6 +262,8 @@ def run_gpu(args):
         else:
             mark(3)
             plan.locate_decode(Z, None, flags, u)
+            if world > 1:      # a node is flagged if any shard saw it disagree
+                merge_flags(flags)
         mark(4)
 
     def sync_all():
@@ -309,7 +310,7 @@ def run_gpu(args):
     # DRAM bytes per gradient coordinate of the dominant kernel, from the ncu captures summarised under profiles/
     # (dram__bytes_read.sum + dram__bytes_write.sum at d = 4 M / 8 M; every byte is touched once, so traffic scales with d).
     # Valid for n = 45 with the configured s only; null for any other shape.
-    traffic_per_coord = {("cyc", 45, 5): 525.5, ("cycp", 45, 5): 353.7, ("rep", 45, 3): 183.0}.get((code, n, s))
+    traffic_per_coord = {("cyc", 45, 5): 525.2, ("cycp", 45, 5): 353.8, ("rep", 45, 3): 183.0}.get((code, n, s))
     traffic = traffic_per_coord * d if traffic_per_coord else None
     stages = {}
     for nm in names:
