@@ -296,8 +296,10 @@ def run_gpu(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
     ms_per_step = total_ms / args.steps
-    stage_ms = {nm: statistics.mean(events[k][i].elapsed_time(events[k][i + 1]) for k in range(args.steps))
-                for i, nm in enumerate(names)}
+    per_step = {nm: [events[k][i].elapsed_time(events[k][i + 1]) for k in range(args.steps)] for i, nm in enumerate(names)}
+    stage_ms = {nm: statistics.mean(v) for nm, v in per_step.items()}
+    stage_min = {nm: min(v) for nm, v in per_step.items()}
+    stage_med = {nm: statistics.median(v) for nm, v in per_step.items()}
 
     ab = algorithmic_bytes(code, n, s, d, len(adv))
     value = ab["coded"] * world / (ms_per_step * 1e-3) / 1e9
@@ -316,8 +318,9 @@ def run_gpu(args):
     for nm in names:
         if stage_ms[nm] > 0 and ab.get(nm, 0) > 0:
             g = ab[nm] / (stage_ms[nm] * 1e-3) / 1e9
-            stages[nm] = {"ms": round(stage_ms[nm], 4), "algorithmic_GB": round(ab[nm] / 1e9, 4),
-                          "GB/s": round(g, 1), "frac_of_peak": round(g / peak, 4)}
+            stages[nm] = {"ms": round(stage_ms[nm], 4), "ms_median": round(stage_med[nm], 4), "ms_min": round(stage_min[nm], 4),
+                          "algorithmic_GB": round(ab[nm] / 1e9, 4), "GB/s": round(g, 1), "frac_of_peak": round(g / peak, 4),
+                          "frac_of_nominal_8TBps": round(g / 8000.0, 4)}
         else:
             stages[nm] = {"ms": round(stage_ms[nm], 4)}
     launches = (1 + len(adv) + (2 if cyc else 0) + 2 + (1 if (cyc and world > 1) else 0)) * args.steps
@@ -364,6 +367,7 @@ def run_gpu(args):
                            "value_is": "bytes of coded gradients (n d complex64 / fp32) per step / step time"},
                 "roofline": {"bound": "hbm", "kernel": dom_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                              "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                             "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
                              "algorithmic_bytes_per_launch": ab[dom], "avg_launch_ms": stage_ms[dom]},
                 "stages": stages, "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "cpu_baseline": cb}
         print(json.dumps(line))

@@ -229,7 +229,7 @@ def test_full_size_resnet152_config_sampled():
     assert sorted(np.flatnonzero(host(flags))) == adv.tolist()            # Lemma 4: V = the corrupted nodes
     assert info["locator_rank"] == s and info["status"] == 0
     rng = np.random.default_rng(2)
-    idx = np.unique(np.concatenate([np.arange(4096), np.arange(d - 4096, d), rng.integers(0, d, 100_000)]))
+    idx = np.unique(np.concatenate([np.arange(4096), np.arange(d - 4096, d), rng.integers(0, d, 1_000_000)]))
     Gs = di.gradient_rows(seed, n, d, idx=idx)
     np.testing.assert_array_equal(host(G[:, idx]), Gs)                     # same inputs on both sides
     # encode on the sample

@@ -158,7 +158,7 @@ def test_full_size_resnet18_config_sampled():
     info = plan.info()
     assert sorted(np.flatnonzero(host(flags))) == adv.tolist() and info["no_majority"] == 0
     rng = np.random.default_rng(1)
-    idx = np.unique(np.concatenate([np.arange(4096), np.arange(d - 4096, d), rng.integers(0, d, 200_000)]))
+    idx = np.unique(np.concatenate([np.arange(4096), np.arange(d - 4096, d), rng.integers(0, d, 1_000_000)]))
     Gs = di.gradient_rows(seed, n, d, 0.0, 0.1, idx=idx)
     np.testing.assert_array_equal(host(G[:, idx]), Gs)                      # same inputs on both sides
     Rs = orc.rep_encode(Gs, n, s)
