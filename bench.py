@@ -169,13 +169,13 @@ class ClockSampler:
         try:
             self.fh = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.fh,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.fh,
                                          stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_min_mhz": None, "sm_max_mhz": None, "power_w_max": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -184,7 +184,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.fh.close()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         try:
             for ln in open(self.path):
                 p = [x.strip() for x in ln.split(",")]
@@ -195,6 +195,10 @@ class ClockSampler:
                     mx.append(float(p[2]))
                 except ValueError:
                     continue
+                try:
+                    pw.append(float(p[3]))
+                except ValueError:
+                    pass
                 for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
                     if val.lower().startswith("active"):
                         reasons.add(name)
@@ -202,7 +206,9 @@ class ClockSampler:
         except Exception:
             pass
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_min_mhz=min(sm), sm_max_mhz=max(mx), samples=len(sm))
+        if pw:
+            out["power_w_max"] = max(pw)
         out["reasons"] = sorted(reasons)
         return out
 
@@ -305,14 +311,14 @@ def run_gpu(args):
     value = ab["coded"] * world / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak_gbs()
     if cyc:
-        dom, dom_kernel = "encode", f"cyc_encode_ring_kernel<S={s}, packed={str(packed).lower()}>"
+        dom, dom_kernel = "encode", f"cyc_encode_stream_kernel<S={s}, packed={str(packed).lower()}>"
     else:
         dom, dom_kernel = "decode", "rep_vote_kernel"
     achieved = ab[dom] / (stage_ms[dom] * 1e-3) / 1e9
     # DRAM bytes per gradient coordinate of the dominant kernel, from the ncu captures summarised under profiles/
     # (dram__bytes_read.sum + dram__bytes_write.sum at d = 4 M / 8 M; every byte is touched once, so traffic scales with d).
     # Valid for n = 45 with the configured s only; null for any other shape.
-    traffic_per_coord = {("cyc", 45, 5): 525.2, ("cycp", 45, 5): 353.8, ("rep", 45, 3): 183.0}.get((code, n, s))
+    traffic_per_coord = {("cyc", 45, 5): 525.1, ("cycp", 45, 5): 353.6, ("rep", 45, 3): 183.0}.get((code, n, s))
     traffic = traffic_per_coord * d if traffic_per_coord else None
     stages = {}
     for nm in names:

@@ -56,7 +56,8 @@ enum {
     DRACO_ECUDA = -2,    /* a CUDA runtime call failed (see draco_last_cuda_error) */
     DRACO_ETOOMANY = -3, /* more than 2 s nodes flagged: no decode vector exists (u is written as zeros) */
     DRACO_ENOMEM = -4,
-    DRACO_EINTERNAL = -5, /* a bounded wait inside a kernel expired (reported by draco_get_info); results are invalid */
+    DRACO_EINTERNAL = -5, /* a bounded wait inside a kernel expired (reported by draco_get_info); results are invalid.
+                             Kept for ABI stability: the current kernels contain no such wait and never report it */
     DRACO_ELIMIT = -6,   /* a size exceeds a fixed capacity of the entry point called (see draco_cyc_project_noalloc) */
     DRACO_ENOMAJ = 1     /* warning: some (group, coordinate) had no strict majority; u holds Algorithm 2's candidate */
 };
@@ -72,7 +73,8 @@ typedef struct draco_info {
     uint64_t no_majority;  /* repetition: (group, coordinate) pairs without a strict majority */
     double scale;          /* cyclic: median_j |e_j| of the projection, the unit of the threshold */
     double max_syndrome;   /* cyclic: max_m |h_m| over the 2 s syndromes */
-    int32_t internal_error; /* non-zero: a kernel gave up a bounded wait (sticky); draco_get_info then returns DRACO_EINTERNAL */
+    int32_t internal_error; /* non-zero: a kernel gave up a bounded wait (sticky); draco_get_info then returns DRACO_EINTERNAL.
+                               Always 0 with the current kernels, none of which spins on a flag */
     int32_t reserved;
 } draco_info;
 

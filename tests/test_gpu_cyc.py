@@ -285,7 +285,7 @@ def test_full_size_decode_on_generated_R_sampled():
 
 
 # ------------------------------------------------------------------ packed transport (Section 3, last paragraph)
-# (n, s, d): d % 8 == 0 takes the ring kernel and 64-bit stores; the others the generic paths (odd d pads the last imaginary part)
+# (n, s, d): d % 8 == 0 takes the streaming kernel and 64-bit stores; the others the generic paths (odd d pads the last imaginary part)
 PACKED_SHAPES = [(15, 2, 100_000), (45, 5, 24_592), (45, 3, 6152), (15, 2, 1001), (9, 1, 6), (15, 7, 4100), (20, 8, 1032)]
 
 
