@@ -10,6 +10,9 @@ N > 1 (torchrun, one rank per GPU) every rank holds its own d-slice of that size
 the only exchange is one all-reduce of the n complex projections inside the locator.
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
+Besides the contract keys the line carries `stages` (per-stage CUDA-event times), `clocks` (nvidia-smi
+sampled every 20 ms during the timed steps) and `graph_replay` (the same step captured once into a CUDA
+graph and replayed: what the launch overhead costs on small workloads).
 """
 from __future__ import annotations
 
@@ -331,6 +334,33 @@ def run_gpu(args):
             stages[nm] = {"ms": round(stage_ms[nm], 4)}
     launches = (1 + len(adv) + (2 if cyc else 0) + 2 + (1 if (cyc and world > 1) else 0)) * args.steps
 
+    # the same step captured once into a CUDA graph and replayed (one GPU only: the sharded step has a collective)
+    graph_replay = None
+    if world == 1 and not args.no_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        cg = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(cg, stream=side):
+                step()
+        stream.wait_stream(side)
+        for _ in range(3):
+            cg.replay()
+        sync_all()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for _ in range(args.steps):
+            cg.replay()
+        g1.record(stream)
+        sync_all()
+        got = sorted(np.flatnonzero(flags.cpu().numpy()).tolist())
+        if got != adv.tolist():
+            raise SystemExit(f"graph replay: flags {got} differ from the planted adversaries {adv.tolist()}")
+        gms = g0.elapsed_time(g1) / args.steps
+        graph_replay = {"ms_per_step": gms, "value": ab["coded"] / (gms * 1e-3) / 1e9, "unit": UNIT,
+                        "stream_launch_ms_per_step": ms_per_step}
+        del cg
+
     # end to end through the host-buffer entry point (rank-local; H2D of G and f, D2H of u and flags)
     e2e = None
     if not args.no_e2e:
@@ -375,7 +405,8 @@ def run_gpu(args):
                              "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                              "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
                              "algorithmic_bytes_per_launch": ab[dom], "avg_launch_ms": stage_ms[dom]},
-                "stages": stages, "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "cpu_baseline": cb}
+                "stages": stages, "clocks": clocks, "e2e": e2e, "graph_replay": graph_replay, "gpu_launches": launches,
+                "cpu_baseline": cb}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -498,6 +529,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--d", type=int, default=None, help="override the workload's d (profiling on a small case)")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay of the step")
     ap.add_argument("--sweep", action="store_true", help="both codes over n x s x d (one GPU); JSON lines to --sweep-out")
     ap.add_argument("--sweep-codes", default="rep,cyc")
     ap.add_argument("--sweep-n", default="15,45,105")
