@@ -271,44 +271,68 @@ cyc_project_manyrows_kernel(const float2* __restrict__ R, const float* __restric
     }
 }
 
-// e_j = sum over the blocks' partials: one warp per row, lane l takes blocks l, l+32, .., then a
-// butterfly over the lanes.  The order is fixed, so the sum is reproducible bit for bit.
-__device__ __forceinline__ double2 sum_partials_row(const double2* __restrict__ partial, int grid, int n, int j, int lane) {
+// e_j = sum over the blocks' partials, by the whole block.  Thread t takes node j = t mod jp (jp = n rounded up to
+// a multiple of 32, so that a warp reads consecutive nodes of one block: coalesced) and every `groups`-th block
+// starting at block t / jp; the group sums of a node are then added in ascending order.  The order is fixed, so
+// the sum is reproducible bit for bit.  red: shared, blockDim.x entries; e_out: n entries, shared or global,
+// valid after the trailing barrier.
+__device__ __forceinline__ void block_sum_partials(const double2* __restrict__ partial, int grid, int n, double2* red,
+                                                   double2* e_out) {
+    const int tid = threadIdx.x;
+    const int jp = (n + 31) & ~31;
+    const int groups = blockDim.x / jp;                  // >= 4 with 512 threads and n <= 128
+    const int j = tid % jp, g = tid / jp;
     double a = 0.0, b = 0.0;
-    for (int blk = lane; blk < grid; blk += 32) {
-        const double2 p = partial[(int64_t)blk * n + j];
-        a += p.x;
-        b += p.y;
+    if (g < groups && j < n) {
+#pragma unroll 8
+        for (int blk = g; blk < grid; blk += groups) {
+            const double2 p = partial[(int64_t)blk * n + j];
+            a += p.x;
+            b += p.y;
+        }
     }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        a += __shfl_xor_sync(0xffffffffu, a, off);
-        b += __shfl_xor_sync(0xffffffffu, b, off);
+    red[tid] = make_double2(a, b);
+    __syncthreads();
+    if (tid < n) {
+        double x = 0.0, y = 0.0;
+        for (int q = 0; q < groups; ++q) {
+            const double2 p = red[q * jp + tid];
+            x += p.x;
+            y += p.y;
+        }
+        e_out[tid] = make_double2(x, y);
     }
-    return make_double2(a, b);
+    __syncthreads();
 }
 
 __global__ void __launch_bounds__(1024)
 cyc_project_finish_kernel(const double2* __restrict__ partial, int grid, int n, double2* e) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    for (int j = warp; j < n; j += nwarps) {
-        const double2 v = sum_partials_row(partial, grid, n, j, lane);
-        if (lane == 0) e[j] = v;
-    }
+    __shared__ double2 red[1024];
+    block_sum_partials(partial, grid, n, red, e);
+}
+
+// The small solves below run either on the whole block (WARP = false: block-wide barriers, any size) or on its
+// first warp alone (WARP = true: warp barriers only; the matrices then sit in shared memory).  The arithmetic and
+// its order are the same in both.
+template <bool WARP>
+__device__ __forceinline__ void small_sync() {
+    if (WARP) __syncwarp(); else __syncthreads();
 }
 
 // ------------------------------------------------------------------ small dense solve
 // Gauss-Jordan elimination with complete pivoting on the dim x (dim+1) augmented matrix A
-// (row stride dim+1) by one thread block.  Pivots with |pivot| <= tol end the elimination
-// (numerical rank); the free unknowns are set to zero.  x receives the solution.
+// (row stride dim+1).  Pivots with |pivot| <= tol end the elimination (numerical rank); the
+// free unknowns are set to zero.  x receives the solution.  WARP: called by warp 0 only, dim <= 32.
+template <bool WARP>
 __device__ int block_gauss_jordan(double2* A, int dim, double tol, double2* x, int* perm, double* rowbest,
                                   int* rowbestc, int* sh) {
     const int tid = threadIdx.x, ldA = dim + 1;
-    for (int i = tid; i < dim; i += blockDim.x) perm[i] = i;
-    __syncthreads();
+    const int nthr = WARP ? 32 : blockDim.x;
+    for (int i = tid; i < dim; i += nthr) perm[i] = i;
+    small_sync<WARP>();
     int rank = 0;
     for (int p = 0; p < dim; ++p) {
-        for (int i = p + tid; i < dim; i += blockDim.x) {
+        for (int i = p + tid; i < dim; i += nthr) {
             double best = -1.0;
             int bc = p;
             for (int c = p; c < dim; ++c) {
@@ -318,7 +342,7 @@ __device__ int block_gauss_jordan(double2* A, int dim, double tol, double2* x, i
             rowbest[i] = best;
             rowbestc[i] = bc;
         }
-        __syncthreads();
+        small_sync<WARP>();
         if (tid == 0) {
             double best = -1.0;
             int br = p;
@@ -328,27 +352,27 @@ __device__ int block_gauss_jordan(double2* A, int dim, double tol, double2* x, i
             sh[1] = rowbestc[br];
             sh[2] = (best > tol * tol) ? 1 : 0;
         }
-        __syncthreads();
+        small_sync<WARP>();
         const int pr = sh[0], pc = sh[1], ok = sh[2];
         if (!ok) break;
         if (pr != p)
-            for (int c = tid; c <= dim; c += blockDim.x) {
+            for (int c = tid; c <= dim; c += nthr) {
                 const double2 tmp = A[p * ldA + c];
                 A[p * ldA + c] = A[pr * ldA + c];
                 A[pr * ldA + c] = tmp;
             }
-        __syncthreads();
+        small_sync<WARP>();
         if (pc != p) {
-            for (int i = tid; i < dim; i += blockDim.x) {
+            for (int i = tid; i < dim; i += nthr) {
                 const double2 tmp = A[i * ldA + p];
                 A[i * ldA + p] = A[i * ldA + pc];
                 A[i * ldA + pc] = tmp;
             }
             if (tid == 0) { const int tmp = perm[p]; perm[p] = perm[pc]; perm[pc] = tmp; }
         }
-        __syncthreads();
+        small_sync<WARP>();
         const double2 piv = A[p * ldA + p];
-        for (int i = tid; i < dim; i += blockDim.x) {
+        for (int i = tid; i < dim; i += nthr) {
             if (i == p) continue;
             const double2 factor = cdiv(A[i * ldA + p], piv);
             for (int c = p + 1; c <= dim; ++c) {
@@ -358,14 +382,14 @@ __device__ int block_gauss_jordan(double2* A, int dim, double tol, double2* x, i
             }
             A[i * ldA + p] = make_double2(0.0, 0.0);
         }
-        __syncthreads();
+        small_sync<WARP>();
         rank = p + 1;
     }
-    __syncthreads();
-    for (int i = tid; i < dim; i += blockDim.x) x[i] = make_double2(0.0, 0.0);
-    __syncthreads();
-    for (int k = tid; k < rank; k += blockDim.x) x[perm[k]] = cdiv(A[k * ldA + dim], A[k * ldA + k]);
-    __syncthreads();
+    small_sync<WARP>();
+    for (int i = tid; i < dim; i += nthr) x[i] = make_double2(0.0, 0.0);
+    small_sync<WARP>();
+    for (int k = tid; k < rank; k += nthr) x[perm[k]] = cdiv(A[k * ldA + dim], A[k * ldA + k]);
+    small_sync<WARP>();
     return rank;
 }
 
@@ -380,8 +404,9 @@ __device__ int block_gauss_jordan(double2* A, int dim, double tol, double2* x, i
 __device__ int block_jacobi_pinv(double2* A, double2* V, const double2* rhs, int s, double tol, double2* beta,
                                  double2* coef, int* sh) {
     const int tid = threadIdx.x;
+    const int nthr = blockDim.x;
     const int sp = s + (s & 1);
-    for (int idx = tid; idx < sp * sp; idx += blockDim.x) {
+    for (int idx = tid; idx < sp * sp; idx += nthr) {
         const int c = idx / sp, i = idx % sp;
         V[idx] = make_double2(c == i ? 1.0 : 0.0, 0.0);
     }
@@ -462,27 +487,130 @@ __device__ int block_jacobi_pinv(double2* A, double2* V, const double2* rhs, int
     return sh[1];
 }
 
+
+// The same solve by one warp for s <= 16 (A, V in shared memory): the pairs of a step sit side by side in the
+// warp, LP lanes per pair (a power of two), each lane holding the rows sub, sub + LP, .. of its pair's columns;
+// the three inner products of a pair are reduced with shuffles inside its LP lanes, every lane of the pair then
+// forms the same rotation and applies it to its own rows.  Only warp barriers.  Called by all 32 lanes of warp 0.
+__device__ int warp_jacobi_pinv(double2* A, double2* V, const double2* rhs, int s, double tol, double2* beta,
+                                double2* coef, int* sh) {
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int sp = s + (s & 1), npairs = sp / 2;
+    int lp = 1;
+    while (lp * 2 * npairs <= 32) lp *= 2;
+    const int pair = lane / lp, sub = lane % lp;
+    const bool act = pair < npairs;
+    for (int idx = lane; idx < sp * sp; idx += 32) {
+        const int c = idx / sp, i = idx % sp;
+        V[idx] = make_double2(c == i ? 1.0 : 0.0, 0.0);
+    }
+    __syncwarp();
+    for (int sweep = 0; sweep < 60; ++sweep) {
+        bool rotated = false;
+        for (int step = 0; step < sp - 1; ++step) {
+            int p = 0, q = 1;
+            if (act) {
+                int a, b;
+                if (pair == 0) { a = sp - 1; b = step; }
+                else { a = (step + pair) % (sp - 1); b = (step - pair + (sp - 1)) % (sp - 1); }
+                p = a < b ? a : b;
+                q = a < b ? b : a;
+            }
+            double2* ap = A + p * sp;
+            double2* aq = A + q * sp;
+            double alpha = 0.0, bet = 0.0, gr = 0.0, gi = 0.0;
+            if (act)
+                for (int i = sub; i < s; i += lp) {
+                    const double2 x = ap[i], y = aq[i];
+                    alpha += x.x * x.x + x.y * x.y;
+                    bet += y.x * y.x + y.y * y.y;
+                    gr += x.x * y.x + x.y * y.y;          // conj(x) * y
+                    gi += x.x * y.y - x.y * y.x;
+                }
+            for (int off = lp >> 1; off > 0; off >>= 1) {
+                alpha += __shfl_xor_sync(full, alpha, off);
+                bet += __shfl_xor_sync(full, bet, off);
+                gr += __shfl_xor_sync(full, gr, off);
+                gi += __shfl_xor_sync(full, gi, off);
+            }
+            const double g2 = gr * gr + gi * gi;
+            if (act && g2 > 1e-30 * alpha * bet && g2 > 0.0) {
+                const double g = sqrt(g2);
+                const double2 ph = make_double2(gr / g, -gi / g);      // exp(-i arg gamma)
+                const double zeta = (bet - alpha) / (2.0 * g);
+                const double tt = copysign(1.0, zeta) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+                const double c = 1.0 / sqrt(1.0 + tt * tt), sn = c * tt;
+                for (int i = sub; i < s; i += lp) {
+                    const double2 x = ap[i], y = cmul(aq[i], ph);
+                    ap[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
+                    aq[i] = make_double2(sn * x.x + c * y.x, sn * x.y + c * y.y);
+                }
+                double2* vp = V + p * sp;
+                double2* vq = V + q * sp;
+                for (int i = sub; i < sp; i += lp) {
+                    const double2 x = vp[i], y = cmul(vq[i], ph);
+                    vp[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
+                    vq[i] = make_double2(sn * x.x + c * y.x, sn * x.y + c * y.y);
+                }
+                rotated = true;
+            }
+            __syncwarp();
+        }
+        if (!__any_sync(full, rotated)) break;
+    }
+    bool keep = false;
+    if (lane < sp) {
+        const double2* ak = A + lane * sp;
+        double sig2 = 0.0, pr = 0.0, pi = 0.0;
+        for (int i = 0; i < s; ++i) {
+            const double2 x = ak[i], r = rhs[i];
+            sig2 += x.x * x.x + x.y * x.y;
+            pr += x.x * r.x + x.y * r.y;                  // conj(x) * r
+            pi += x.x * r.y - x.y * r.x;
+        }
+        keep = sqrt(sig2) > tol;
+        coef[lane] = keep ? make_double2(pr / sig2, pi / sig2) : make_double2(0.0, 0.0);
+    }
+    const int rank = __popc(__ballot_sync(full, keep));
+    __syncwarp();
+    if (lane < s) {
+        double re = 0.0, im = 0.0;
+        for (int k = 0; k < sp; ++k) {
+            const double2 q = cmul(V[k * sp + lane], coef[k]);
+            re += q.x;
+            im += q.y;
+        }
+        beta[lane] = make_double2(re, im);
+    }
+    if (lane == 0) sh[1] = rank;
+    __syncwarp();
+    return rank;
+}
+
+constexpr int kSmallDim = 16;         // systems up to this size are solved in shared memory by one warp
+
 // ------------------------------------------------------------------ locator after the projection
 __global__ void __launch_bounds__(kSolveThreads)
 cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ partial, int grid, const double2* __restrict__ e_in,
                  int n, int s, double theta, uint8_t* flags, uint8_t* flags2, DeviceInfo* info) {
-    __shared__ double2 e[kMaxN], h[kMaxN];
+    __shared__ double2 e[kMaxN], h[kMaxN], tw[kMaxN];
+    __shared__ double2 red[kSolveThreads];
+    __shared__ double2 As[kSmallDim * kSmallDim], Vs[kSmallDim * kSmallDim];
+    __shared__ double2 rhs_s[kMaxN / 2], beta_s[kMaxN / 2], coef_s[kMaxN / 2];
     __shared__ double mag[kMaxN], sorted[kMaxN];
     __shared__ int sh[4], count;
     __shared__ double scale_s, maxsyn_s;
     const int tid = threadIdx.x;
     const double rsn = 1.0 / sqrt((double)n);
 
+    if (tid < n) tw[tid] = cd->twiddle[tid];
     if (e_in == nullptr) {
-        const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
-        for (int j = warp; j < n; j += nwarps) {
-            const double2 v = sum_partials_row(partial, grid, n, j, lane);
-            if (lane == 0) e[j] = v;
-        }
-    } else if (tid < n) {
-        e[tid] = e_in[tid];
+        block_sum_partials(partial, grid, n, red, e);
+    } else {
+        if (tid < n) e[tid] = e_in[tid];
+        __syncthreads();
     }
-    __syncthreads();
     if (tid < n) {
         const double2 v = e[tid];
         cd->e[tid] = v;
@@ -503,10 +631,13 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ partial, int grid, c
     if (tid < 2 * s) {
         const int m = n - 2 * s + tid;
         double a = 0.0, b = 0.0;
+        int idx = 0;                                       // (m j) mod n
         for (int j = 0; j < n; ++j) {
-            const double2 q = cmulc(e[j], cd->twiddle[(m * j) % n]);
+            const double2 q = cmulc(e[j], tw[idx]);
             a += q.x;
             b += q.y;
+            idx += m;
+            if (idx >= n) idx -= n;
         }
         h[m] = make_double2(a * rsn, b * rsn);
     }
@@ -520,24 +651,28 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ partial, int grid, c
     const double tol = theta * scale_s;
     int rank = 0;
     bool flagged = false;
+    double2* beta = beta_s;
     if (s > 0) {
         // row i: [h_{n-s-1-i} .. h_{n-2-i}] beta = h_{n-1-i}; stored by columns
         const int sp = s + (s & 1);
-        double2* A = cd->work;
-        double2* V = cd->work + sp * sp;
-        double2* rhs = cd->vec;
-        double2* beta = cd->vec + kMaxN;
-        double2* coef = cd->vec + 2 * kMaxN;
+        const bool small = sp <= kSmallDim;
+        double2* A = small ? As : cd->work;
+        double2* V = small ? Vs : cd->work + sp * sp;
         for (int idx = tid; idx < sp * sp; idx += blockDim.x) {
             const int c = idx / sp, i = idx % sp;
             A[idx] = (c < s && i < s) ? h[n - s - 1 - i + c] : make_double2(0.0, 0.0);
         }
-        if (tid < s) rhs[tid] = h[n - 1 - tid];
+        if (tid < s) rhs_s[tid] = h[n - 1 - tid];
         __syncthreads();
-        rank = block_jacobi_pinv(A, V, rhs, s, tol, beta, coef, sh);
+        if (small) {
+            if (tid < 32) warp_jacobi_pinv(A, V, rhs_s, s, tol, beta_s, coef_s, sh);
+            __syncthreads();
+            rank = sh[1];
+        } else {
+            rank = block_jacobi_pinv(A, V, rhs_s, s, tol, beta_s, coef_s, sh);
+        }
     }
     if (rank > 0) {
-        double2* beta = cd->vec + kMaxN;
         if (tid == 0) {
             for (int l = 0; l < n - 2 * s; ++l) {
                 double a = 0.0, b = 0.0;
@@ -554,10 +689,13 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ partial, int grid, c
         __syncthreads();
         if (tid < n) {
             double a = 0.0, b = 0.0;
+            int idx = 0;                                   // (tid m) mod n
             for (int m = 0; m < n; ++m) {
-                const double2 q = cmul(h[m], cd->twiddle[(tid * m) % n]);
+                const double2 q = cmul(h[m], tw[idx]);
                 a += q.x;
                 b += q.y;
+                idx += tid;
+                if (idx >= n) idx -= n;
             }
             const double2 t = make_double2(a * rsn, b * rsn);
             cd->t[tid] = t;
@@ -596,16 +734,23 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ partial, int grid, c
 // I - B^H B = [C_R]_{.,V}^H [C_R]_{.,V} is only |V| x |V| (|V| <= 2 s).
 __global__ void __launch_bounds__(kSolveThreads)
 cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n, int s, DeviceInfo* info) {
-    __shared__ int vlist[kMaxN], rowbestc[kMaxN], sh[4], a_s;
+    __shared__ int vlist[kMaxN], rowbestc[kMaxN], perm_s[kMaxN], sh[4], a_s;
+    __shared__ uint8_t fl[kMaxN];
     __shared__ double rowbest[kMaxN];
-    __shared__ double2 y[kMaxN];
+    __shared__ double2 y[kMaxN], tw[kMaxN], x_s[kMaxN], b_s[kMaxN];
+    __shared__ double2 As[kSmallDim * (kSmallDim + 1)];
     const int tid = threadIdx.x;
     const int rows = n - 2 * s, L = rows - 1;
     const double rsn = 1.0 / sqrt((double)n);
+    if (tid < n) {
+        tw[tid] = cd->twiddle[tid];
+        fl[tid] = flags[tid];
+    }
+    __syncthreads();
     if (tid == 0) {
         int a = 0;
         for (int j = 0; j < n; ++j)
-            if (flags[j]) vlist[a++] = j;
+            if (fl[j]) vlist[a++] = j;
         a_s = a;
     }
     __syncthreads();
@@ -615,9 +760,10 @@ cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n
         if (tid == 0) { info->n_active = 0; info->n_flagged = a; info->status = DRACO_ETOOMANY; }
         return;
     }
-    double2* x = cd->vec;
+    double2* x = x_s;
     if (a > 0) {
-        double2* A = cd->work;
+        const bool small = a <= kSmallDim;
+        double2* A = small ? As : cd->work;
         for (int idx = tid; idx < a * (a + 1); idx += blockDim.x) {
             const int p = idx / (a + 1), q = idx % (a + 1);
             double2 val;
@@ -625,25 +771,33 @@ cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n
                 int dv = vlist[q] - vlist[p];
                 if (dv < 0) dv += n;
                 double re = 0.0, im = 0.0;
+                int k = ((n - 2 * s) * dv) % n;
                 for (int m = n - 2 * s; m < n; ++m) {
-                    const double2 w = cd->twiddle[(m * dv) % n];
+                    const double2 w = tw[k];
                     re += w.x;
                     im += w.y;
+                    k += dv;
+                    if (k >= n) k -= n;
                 }
                 val = make_double2(re / n, im / n);
             } else {                                       // conj(C[L][v_p])
-                const double2 w = cd->twiddle[(L * vlist[p]) % n];
+                const double2 w = tw[(L * vlist[p]) % n];
                 val = make_double2(w.x * rsn, -w.y * rsn);
             }
             A[idx] = val;
         }
         __syncthreads();
-        block_gauss_jordan(A, a, 0.0, x, cd->perm, rowbest, rowbestc, sh);
+        if (small) {
+            if (tid < 32) block_gauss_jordan<true>(A, a, 0.0, x, perm_s, rowbest, rowbestc, sh);
+            __syncthreads();
+        } else {
+            block_gauss_jordan<false>(A, a, 0.0, x, perm_s, rowbest, rowbestc, sh);
+        }
     }
     if (tid < rows) {
         double re = (tid == L) ? 1.0 : 0.0, im = 0.0;
         for (int p = 0; p < a; ++p) {
-            const double2 w = cd->twiddle[(tid * vlist[p]) % n];
+            const double2 w = tw[(tid * vlist[p]) % n];
             const double2 q = cmul(w, x[p]);
             re += q.x * rsn;
             im += q.y * rsn;
@@ -653,27 +807,31 @@ cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n
     __syncthreads();
     if (tid < n) {
         double2 b = make_double2(0.0, 0.0);
-        if (!flags[tid]) {
+        if (!fl[tid]) {
             double re = 0.0, im = 0.0;
+            int k = 0;                                     // (m tid) mod n
             for (int m = 0; m < rows; ++m) {
-                const double2 q = cmulc(y[m], cd->twiddle[(m * tid) % n]);
+                const double2 q = cmulc(y[m], tw[k]);
                 re += q.x;
                 im += q.y;
+                k += tid;
+                if (k >= n) k -= n;
             }
             b = make_double2(re * rsn, im * rsn);
         }
         cd->b[tid] = b;
+        b_s[tid] = b;
     }
     __syncthreads();
-    if (tid == 0) {
+    // the active rows in ascending order: position = number of unflagged nodes before this one
+    if (tid < n && !fl[tid]) {
         int k = 0;
-        for (int j = 0; j < n; ++j)
-            if (!flags[j]) {
-                cd->active[k] = j;
-                cd->b_active[k] = cd->b[j];
-                ++k;
-            }
-        info->n_active = k;
+        for (int j = 0; j < tid; ++j) k += fl[j] ? 0 : 1;
+        cd->active[k] = tid;
+        cd->b_active[k] = b_s[tid];
+    }
+    if (tid == 0) {
+        info->n_active = n - a;
         info->n_flagged = a;
         if (info->status == DRACO_ETOOMANY) info->status = DRACO_OK;
     }
