@@ -248,7 +248,7 @@ def run_gpu(args):
     Z = torch.empty((n, (2 if cyc else 1) * vlen), dtype=torch.float32, device="cuda")
     u = torch.empty(d, dtype=torch.float32, device="cuda")
     flags = torch.empty(n, dtype=torch.uint8, device="cuda")
-    e = torch.empty(2 * n, dtype=torch.float64, device="cuda")
+    e = torch.empty(3 * n, dtype=torch.float64, device="cuda")        # projection record: n (re, im) pairs + n squared norms
 
     names = ["encode", "corrupt", "locate", "decode"]
 
@@ -262,7 +262,7 @@ def run_gpu(args):
         plan.corrupt(Z, adv, model, param, seed=SEED + 2)
         mark(2)
         if cyc:
-            if world > 1:      # d-sharded: local projection, all-reduce of the 2 n doubles, local solve
+            if world > 1:      # d-sharded: local projection, all-reduce of the 3 n doubles, local solve
                 locate_sharded(plan, Z, f, flags, e)
             else:
                 plan.locate(Z, f, flags)

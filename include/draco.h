@@ -71,7 +71,7 @@ typedef struct draco_info {
     int32_t locator_rank;  /* cyclic: numerical rank of the s x s syndrome system = adversaries seen */
     int32_t n_active;      /* cyclic decode: number of rows with b_j != 0 */
     uint64_t no_majority;  /* repetition: (group, coordinate) pairs without a strict majority */
-    double scale;          /* cyclic: median_j |e_j| of the projection, the unit of the threshold */
+    double scale;          /* cyclic: median_j q_j^(1/2), q_j = sum_i |R[j][i]|^2: the unit of the rank cutoff */
     double max_syndrome;   /* cyclic: max_m |h_m| over the 2 s syndromes */
     int32_t internal_error; /* non-zero: a kernel gave up a bounded wait (sticky); draco_get_info then returns DRACO_EINTERNAL.
                                Always 0 with the current kernels, none of which spins on a flag */
@@ -91,9 +91,11 @@ int draco_plan_create(int n, int s, int64_t d, int code, draco_plan** out);
 int draco_plan_destroy(draco_plan* plan);
 
 /* Rank cutoff theta of the cyclic locator (default 1e-6): singular values of the s x s syndrome
- * system below theta * median_j |e_j| count as zero.  The rank found is the number of adversaries
- * seen, and V is the set of that many nodes with the largest |t_j| (exactly that many t_j are
- * non-zero in exact arithmetic). */
+ * system below theta * median_j q_j^(1/2) count as zero, q_j = sum_i |R[j][i]|^2 (the size of what
+ * node j sent: complex64 rounding perturbs e_j by about 2^-25 (2 q_j)^(1/2) even where e_j itself
+ * cancels to something small; the paper's "t_j != 0" needs such a yardstick and names none).
+ * The rank found is the number of adversaries seen, and V is the set of that many nodes with the
+ * largest |t_j| (exactly that many t_j are non-zero in exact arithmetic). */
 int draco_plan_set_theta(draco_plan* plan, double theta);
 
 /* Number of groups of a repetition plan (0 for a cyclic plan); group g covers
@@ -152,7 +154,9 @@ int draco_locate_decode(draco_plan* plan, const void* R, const float* f, uint8_t
 int draco_rep_vote(draco_plan* plan, const void* R, float* u, float* maj, uint8_t* flags, void* stream);
 
 /* The two halves of the cyclic locator, for callers that shard d across devices and add the
- * projections: e (device [n] complex as (re, im) doubles) = f R over this plan's d coordinates. */
+ * projection records.  e: device, 3 n doubles, 16-byte aligned: e_j = (f R)_j as n (re, im) pairs, then the
+ * n values q_j = sum_i |R[j][i]|^2 that set the rank cutoff; both are sums over this plan's d
+ * coordinates, so records of disjoint coordinate ranges add up. */
 int draco_cyc_project(draco_plan* plan, const void* R, const float* f, double* e, void* stream);
 int draco_cyc_locate_from_projection(draco_plan* plan, const double* e, uint8_t* flags, void* stream);
 
@@ -165,11 +169,12 @@ int draco_cyc_locate_from_projection(draco_plan* plan, const double* e, uint8_t*
  * splits the pool), or a step loop that cannot tolerate the device-wide synchronisation that an
  * allocation or free may imply.  draco_plan_create allocates; this entry point needs no plan and
  * calls neither cudaMalloc nor cudaFree nor any allocating library routine.  Its only scratch, the
- * per-block partial sums, is a fixed array compiled into the library: 296 blocks x 128 nodes x 16
- * bytes = 592 KB of device memory on every GPU that loads the library, held until the process ends.
+ * per-block partial sums, is a fixed array compiled into the library: 296 blocks x 128 nodes x 24
+ * bytes = 888 KB of device memory on every GPU that loads the library, held until the process ends.
  *
- * n nodes, d coordinates; R: device [n][d] complex64; f: device [d] fp32; e: device [n] complex as
- * (re, im) doubles, written by the call.  All three 16-byte aligned; the caller owns them.
+ * n nodes, d coordinates; R: device [n][d] complex64; f: device [d] fp32; e: device, 3 n doubles (the
+ * projection record of draco_cyc_project: n (re, im) pairs, then n values q_j), written by the call.
+ * All three 16-byte aligned; the caller owns them.
  * Limits: n <= DRACO_MAX_N (128) and device ordinal < 64, else DRACO_ELIMIT; d is unbounded
  * (at most 296 blocks are launched, each walking its share of the tiles).
  * The first call on each device looks up the array's device address (with that device current);

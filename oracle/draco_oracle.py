@@ -244,9 +244,21 @@ def cyc_project(R: np.ndarray, f: np.ndarray) -> np.ndarray:
     return np.asarray(R, dtype=np.complex128) @ np.asarray(f, dtype=np.float64)
 
 
-def cyc_locate_from_projection(e: np.ndarray, n: int, s: int, theta: float = 1e-6) -> dict:
+def cyc_project_energy(R: np.ndarray) -> np.ndarray:
+    """q_j = sum_i |R[j][i]|^2: the squared size of what node j sent.
+
+    Not in the paper.  Rounding R to complex64 perturbs e_j = sum_i f_i R[j][i] by about
+    2^-25 (E f^2 q_j)^(1/2), E f^2 = 2, whatever e_j itself comes to (the terms of e_j can
+    cancel, those of q_j cannot), so q_j^(1/2) is the yardstick for "zero" in the rank
+    decision of the locator.
+    """
+    R = np.asarray(R, dtype=np.complex128)
+    return np.sum(R.real ** 2 + R.imag ** 2, axis=1)
+
+
+def cyc_locate_from_projection(e: np.ndarray, q: np.ndarray, n: int, s: int, theta: float = 1e-6) -> dict:
     """The locator phi after the projection: syndromes, Toeplitz solve,
-    recurrence, IDFT, support.
+    recurrence, IDFT, support.  e = f R, q = cyc_project_energy(R).
 
     Readings where the paper is garbled or silent:
       * syndromes are h_m, m = n-2s .. n-1 ascending: [h_m] = e C_R^dagger;
@@ -255,16 +267,18 @@ def cyc_locate_from_projection(e: np.ndarray, n: int, s: int, theta: float = 1e-
         l = n-1-i;
       * fewer than s adversaries make the system singular (its rank is the
         number of non-zero entries of gamma = (f N)^T): singular values below
-        theta * scale, scale = median_j |e_j|, count as zero and beta is the
+        theta * scale, scale = median_j q_j^(1/2), count as zero and beta is the
         pseudo-inverse solution; Lemma 8 lets any solution of the equations
-        drive the recurrence;
+        drive the recurrence.  (scale = median_j |e_j| was the first choice; e_j is
+        a signed sum and can cancel to a tenth of its usual size, and with it the
+        cutoff sinks into the rounding noise of complex64 vectors);
       * "t_j != 0" cannot be tested in floating point.  Exactly ``rank`` entries
         of t are non-zero in exact arithmetic, so V = the ``rank`` nodes with the
         largest |t_j| (V is empty when the rank is 0).
     """
     e = np.asarray(e, dtype=np.complex128)
     C = idft_matrix(n)
-    scale = float(np.median(np.abs(e)))
+    scale = float(np.median(np.sqrt(np.asarray(q, dtype=np.float64))))
     tol = theta * scale
     out = {"e": e, "scale": scale, "t": np.zeros(n, dtype=np.complex128),
            "flags": np.zeros(n, dtype=bool), "rank": 0, "h": np.zeros(n, dtype=np.complex128),
@@ -306,7 +320,7 @@ def cyc_locate_from_projection(e: np.ndarray, n: int, s: int, theta: float = 1e-
 
 def cyc_locate(R: np.ndarray, f: np.ndarray, n: int, s: int, theta: float = 1e-6) -> dict:
     """V = phi(R) with the random vector f passed in (f ~ N(1_d, I_d))."""
-    return cyc_locate_from_projection(cyc_project(R, f), n, s, theta)
+    return cyc_locate_from_projection(cyc_project(R, f), cyc_project_energy(R), n, s, theta)
 
 
 def cyc_decode_vector(n: int, s: int, flags) -> np.ndarray:

@@ -35,17 +35,49 @@ __device__ __forceinline__ double2 cdiv(double2 a, double2 b) {
 __device__ __forceinline__ double cabs2(double2 a) { return a.x * a.x + a.y * a.y; }
 
 // ------------------------------------------------------------------ projection
-// Block = 8 warps over one tile of coordinates; warp w owns rows w, w+8, ...; f for the tile
-// sits in shared memory.  Products and short runs (16 terms) in fp32, running sums in fp64.
+// q_j = sum_i |R[j][i]|^2 travels with e_j: it is the yardstick of the locator's rank cutoff (rounding R to
+// complex64 perturbs e_j by about 2^-25 (E f^2 q_j)^(1/2), whatever e_j itself cancels to).  A few digits of it
+// are enough: fp32 terms and tile sums, fp64 across tiles.  Layout of the block partials: [grid][n] double2 (e),
+// then [grid][n] double (q).
+__device__ __forceinline__ float energy2(float4 v, float acc) {
+    acc = fmaf(v.x, v.x, acc);
+    acc = fmaf(v.y, v.y, acc);
+    acc = fmaf(v.z, v.z, acc);
+    return fmaf(v.w, v.w, acc);
+}
+__device__ __forceinline__ double warp_sum(double a) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+    return a;
+}
+__device__ __forceinline__ float warp_sum(float a) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+    return a;
+}
+__device__ __forceinline__ double* q_partials(double2* partial, int n) {
+    return reinterpret_cast<double*>(partial + (int64_t)gridDim.x * n);
+}
+// Block = 8 warps over one tile of coordinates; warp w owns rows row0 + w, row0 + w + 8, ... of the
+// launch's nrows <= 8 RPW rows; f for the tile sits in shared memory.  Products and short runs (16 terms)
+// in fp32, running sums in fp64.  More than 64 rows take two launches of half the rows each (rows are
+// independent; f is read twice, 1 % more traffic): 16 rows per warp in registers halve the blocks per SM
+// (0.79 of the copy bandwidth at n = 105), and per-lane sums in shared memory left the compiler too few
+// registers to keep its loads in flight once the squared norms were added (0.98 -> 0.68).
 template <int RPW, bool VEC2>
 __global__ void __launch_bounds__(kThreads)
 cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
-                   double2* __restrict__ partial, int accumulate) {
+                   int row0, int nrows, double2* __restrict__ partial, int accumulate) {
     __shared__ __align__(16) float fs[kProjectTile];
+    __shared__ double qs[kProjectWarps * RPW];           // q of row warp + r * 8, kept by lane 0 of its warp
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     double accr[RPW], acci[RPW];
 #pragma unroll
     for (int r = 0; r < RPW; ++r) { accr[r] = 0.0; acci[r] = 0.0; }
+    if (lane == 0) {
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) qs[r * kProjectWarps + warp] = 0.0;
+    }
 
     const int64_t ntiles = (len + kProjectTile - 1) / kProjectTile;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
@@ -55,9 +87,10 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
         __syncthreads();
 #pragma unroll
         for (int r = 0; r < RPW; ++r) {
-            const int j = warp + r * kProjectWarps;
-            if (j < n) {
+            const int j = row0 + warp + r * kProjectWarps;
+            if (j < row0 + nrows) {
                 const float2* row = R + (int64_t)j * ld + c0;
+                float eq = 0.f;
                 if (VEC2 && cnt == kProjectTile) {
                     const float4* row4 = reinterpret_cast<const float4*>(row);
 #pragma unroll 1
@@ -65,15 +98,17 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
                         float4 v[8];
 #pragma unroll
                         for (int q = 0; q < 8; ++q) v[q] = __ldcs(row4 + (step0 + q) * 32 + lane);
-                        float pr = 0.f, pi = 0.f;
+                        float pr = 0.f, pi = 0.f, pq = 0.f;
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
                             const float2 ff = *reinterpret_cast<const float2*>(&fs[((step0 + q) * 32 + lane) * 2]);
                             pr = fmaf(ff.x, v[q].x, pr); pi = fmaf(ff.x, v[q].y, pi);
                             pr = fmaf(ff.y, v[q].z, pr); pi = fmaf(ff.y, v[q].w, pi);
+                            pq = energy2(v[q], pq);
                         }
                         accr[r] += (double)pr;
                         acci[r] += (double)pi;
+                        eq += pq;
                     }
                 } else {
                     for (int i = lane; i < cnt; i += 32) {
@@ -81,12 +116,16 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
                         const float ff = fs[i];
                         accr[r] += (double)(ff * v.x);
                         acci[r] += (double)(ff * v.y);
+                        eq = fmaf(v.y, v.y, fmaf(v.x, v.x, eq));
                     }
                 }
+                eq = warp_sum(eq);
+                if (lane == 0) qs[r * kProjectWarps + warp] += (double)eq;
             }
         }
         __syncthreads();
     }
+    double* qpartial = q_partials(partial, n);
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {
         double a = accr[r], b = acci[r];
@@ -95,11 +134,14 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
             a += __shfl_xor_sync(0xffffffffu, a, off);
             b += __shfl_xor_sync(0xffffffffu, b, off);
         }
-        const int j = warp + r * kProjectWarps;
-        if (lane == 0 && j < n) {
+        const int j = row0 + warp + r * kProjectWarps;
+        if (lane == 0 && j < row0 + nrows) {
             double2* dst = partial + (int64_t)blockIdx.x * n + j;
-            if (accumulate) { a += dst->x; b += dst->y; }
+            double* qdst = qpartial + (int64_t)blockIdx.x * n + j;
+            double c = qs[r * kProjectWarps + warp];
+            if (accumulate) { a += dst->x; b += dst->y; c += *qdst; }
             *dst = make_double2(a, b);
+            *qdst = c;
         }
     }
 }
@@ -109,15 +151,17 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
 // of all n rows, with f for its chunk in registers (8 values per lane) and no shared memory or
 // barrier in the loop.  Per-lane running sums in fp64 registers (2 n doubles).
 template <bool VEC2>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)
 cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
                            double2* __restrict__ partial, int accumulate) {
     constexpr int NMAX = 16, CH = 256;
     __shared__ double2 wsum[kProjectWarps][NMAX];
+    __shared__ double wq[kProjectWarps][NMAX];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     double accr[NMAX], acci[NMAX];
+    float accq[NMAX];                                    // q needs a few digits only: fp32 running sums
 #pragma unroll
-    for (int j = 0; j < NMAX; ++j) { accr[j] = 0.0; acci[j] = 0.0; }
+    for (int j = 0; j < NMAX; ++j) { accr[j] = 0.0; acci[j] = 0.0; accq[j] = 0.f; }
     const int64_t nchunks = (len + CH - 1) / CH;
     const int64_t nwarps = (int64_t)gridDim.x * kProjectWarps;
     for (int64_t chunk = (int64_t)blockIdx.x * kProjectWarps + warp; chunk < nchunks; chunk += nwarps) {
@@ -140,23 +184,27 @@ cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict
 #pragma unroll
                         for (int q = 0; q < 4; ++q) vb[q] = __ldcs(rb + q * 32 + lane);
                     }
-                    float pr = 0.f, pi = 0.f;
+                    float pr = 0.f, pi = 0.f, pq = accq[jj];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         pr = fmaf(ff[q].x, va[q].x, pr); pi = fmaf(ff[q].x, va[q].y, pi);
                         pr = fmaf(ff[q].y, va[q].z, pr); pi = fmaf(ff[q].y, va[q].w, pi);
+                        pq = energy2(va[q], pq);
                     }
                     accr[jj] += (double)pr;
                     acci[jj] += (double)pi;
+                    accq[jj] = pq;
                     if (two) {
-                        pr = 0.f; pi = 0.f;
+                        pr = 0.f; pi = 0.f; pq = accq[jj + 1];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             pr = fmaf(ff[q].x, vb[q].x, pr); pi = fmaf(ff[q].x, vb[q].y, pi);
                             pr = fmaf(ff[q].y, vb[q].z, pr); pi = fmaf(ff[q].y, vb[q].w, pi);
+                            pq = energy2(vb[q], pq);
                         }
                         accr[jj + 1] += (double)pr;
                         acci[jj + 1] += (double)pi;
+                        accq[jj + 1] = pq;
                     }
                 }
             }
@@ -169,6 +217,7 @@ cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict
                         const float2 v = __ldcs(R + (int64_t)j * ld + c0 + i);
                         accr[j] += (double)(fi * v.x);
                         acci[j] += (double)(fi * v.y);
+                        accq[j] = fmaf(v.y, v.y, fmaf(v.x, v.x, accq[j]));
                     }
             }
         }
@@ -181,134 +230,69 @@ cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict
             a += __shfl_xor_sync(0xffffffffu, a, off);
             b += __shfl_xor_sync(0xffffffffu, b, off);
         }
-        if (lane == 0) wsum[warp][j] = make_double2(a, b);
+        const double c = warp_sum((double)accq[j]);
+        if (lane == 0) { wsum[warp][j] = make_double2(a, b); wq[warp][j] = c; }
     }
     __syncthreads();
     if (threadIdx.x < n) {
-        double a = 0.0, b = 0.0;
+        double a = 0.0, b = 0.0, c = 0.0;
         for (int w = 0; w < kProjectWarps; ++w) {            // fixed order: reproducible
             a += wsum[w][threadIdx.x].x;
             b += wsum[w][threadIdx.x].y;
+            c += wq[w][threadIdx.x];
         }
         double2* dst = partial + (int64_t)blockIdx.x * n + threadIdx.x;
-        if (accumulate) { a += dst->x; b += dst->y; }
+        double* qdst = q_partials(partial, n) + (int64_t)blockIdx.x * n + threadIdx.x;
+        if (accumulate) { a += dst->x; b += dst->y; c += *qdst; }
         *dst = make_double2(a, b);
+        *qdst = c;
     }
 }
 
-// The same projection for many rows per warp (n > 64): the per-lane running sums live in shared
-// memory instead of registers (2 doubles per row and lane would cost 4 * ceil(n / 8) registers and
-// halve the blocks per SM).  Dynamic shared memory: f tile, then sums[ceil(n / 8)][256] double2.
-template <bool VEC2>
-__global__ void __launch_bounds__(kThreads)
-cyc_project_manyrows_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
-                            double2* __restrict__ partial, int accumulate) {
-    extern __shared__ __align__(16) unsigned char proj_smem[];
-    float* fs = reinterpret_cast<float*>(proj_smem);
-    double2* sums = reinterpret_cast<double2*>(proj_smem + sizeof(float) * kProjectTile);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rpw = (n + kProjectWarps - 1) / kProjectWarps;
-    for (int r = 0; r < rpw; ++r) sums[r * kThreads + threadIdx.x] = make_double2(0.0, 0.0);
-
-    const int64_t ntiles = (len + kProjectTile - 1) / kProjectTile;
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const int64_t c0 = tile * kProjectTile;
-        const int cnt = (int)((len - c0) < kProjectTile ? (len - c0) : kProjectTile);
-        for (int i = threadIdx.x; i < kProjectTile; i += kThreads) fs[i] = (i < cnt) ? __ldcs(f + c0 + i) : 0.0f;
-        __syncthreads();
-        for (int r = 0; r < rpw; ++r) {
-            const int j = warp + r * kProjectWarps;
-            if (j < n) {
-                const float2* row = R + (int64_t)j * ld + c0;
-                double ar = 0.0, ai = 0.0;
-                if (VEC2 && cnt == kProjectTile) {
-                    const float4* row4 = reinterpret_cast<const float4*>(row);
-#pragma unroll 1
-                    for (int step0 = 0; step0 < kProjectTile / 64; step0 += 8) {
-                        float4 v[8];
+// e_j and q_j = sums over the blocks' partials: one block of 128 threads per node j.  Thread t adds the partials
+// of blocks t, t + 128, .. in ascending order, the 128 thread sums are then added by a butterfly inside each warp
+// and the four warp sums in ascending order.  The order is fixed, so the sums are reproducible bit for bit.
+// record: n (re, im) pairs, then n values q_j (3 n doubles).  (A single block doing this for all nodes took
+// 20-40 us: one SM's load latency, serialised.)
+constexpr int kReduceThreads = 128;
+__global__ void __launch_bounds__(kReduceThreads)
+cyc_reduce_partials_kernel(const double2* __restrict__ partial, int grid, int n, double* __restrict__ record) {
+    constexpr int kBatch = 8;
+    __shared__ double wsum[3][kReduceThreads / 32];
+    const int j = blockIdx.x, tid = threadIdx.x;
+    const double* __restrict__ qpartial = reinterpret_cast<const double*>(partial + (int64_t)grid * n);
+    double a = 0.0, b = 0.0, c = 0.0;
+    for (int base = 0; base < grid; base += kBatch * kReduceThreads) {
+        double2 pe[kBatch];
+        double pq[kBatch];
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) v[q] = __ldcs(row4 + (step0 + q) * 32 + lane);
-                        float pr = 0.f, pi = 0.f;
+        for (int u = 0; u < kBatch; ++u) {               // all loads first (beyond the grid: block 0 again, not added)
+            const int blk = base + u * kReduceThreads + tid;
+            const int64_t at = (int64_t)(blk < grid ? blk : 0) * n + j;
+            pe[u] = __ldcg(partial + at);
+            pq[u] = __ldcg(qpartial + at);
+        }
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            const float2 ff = *reinterpret_cast<const float2*>(&fs[((step0 + q) * 32 + lane) * 2]);
-                            pr = fmaf(ff.x, v[q].x, pr); pi = fmaf(ff.x, v[q].y, pi);
-                            pr = fmaf(ff.y, v[q].z, pr); pi = fmaf(ff.y, v[q].w, pi);
-                        }
-                        ar += (double)pr;
-                        ai += (double)pi;
-                    }
-                } else {
-                    for (int i = lane; i < cnt; i += 32) {
-                        const float2 v = __ldcs(row + i);
-                        const float ff = fs[i];
-                        ar += (double)(ff * v.x);
-                        ai += (double)(ff * v.y);
-                    }
-                }
-                double2 s = sums[r * kThreads + threadIdx.x];      // this thread's own slot: no synchronisation needed
-                s.x += ar;
-                s.y += ai;
-                sums[r * kThreads + threadIdx.x] = s;
+        for (int u = 0; u < kBatch; ++u) {
+            if (base + u * kReduceThreads + tid < grid) {
+                a += pe[u].x;
+                b += pe[u].y;
+                c += pq[u];
             }
         }
-        __syncthreads();
     }
-    for (int r = 0; r < rpw; ++r) {
-        const double2 s = sums[r * kThreads + threadIdx.x];
-        double a = s.x, b = s.y;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            a += __shfl_xor_sync(0xffffffffu, a, off);
-            b += __shfl_xor_sync(0xffffffffu, b, off);
-        }
-        const int j = warp + r * kProjectWarps;
-        if (lane == 0 && j < n) {
-            double2* dst = partial + (int64_t)blockIdx.x * n + j;
-            if (accumulate) { a += dst->x; b += dst->y; }
-            *dst = make_double2(a, b);
-        }
-    }
-}
-
-// e_j = sum over the blocks' partials, by the whole block.  Thread t takes node j = t mod jp (jp = n rounded up to
-// a multiple of 32, so that a warp reads consecutive nodes of one block: coalesced) and every `groups`-th block
-// starting at block t / jp; the group sums of a node are then added in ascending order.  The order is fixed, so
-// the sum is reproducible bit for bit.  red: shared, blockDim.x entries; e_out: n entries, shared or global,
-// valid after the trailing barrier.
-__device__ __forceinline__ void block_sum_partials(const double2* __restrict__ partial, int grid, int n, double2* red,
-                                                   double2* e_out) {
-    const int tid = threadIdx.x;
-    const int jp = (n + 31) & ~31;
-    const int groups = blockDim.x / jp;                  // >= 4 with 512 threads and n <= 128
-    const int j = tid % jp, g = tid / jp;
-    double a = 0.0, b = 0.0;
-    if (g < groups && j < n) {
-#pragma unroll 8
-        for (int blk = g; blk < grid; blk += groups) {
-            const double2 p = partial[(int64_t)blk * n + j];
-            a += p.x;
-            b += p.y;
-        }
-    }
-    red[tid] = make_double2(a, b);
+    a = warp_sum(a);
+    b = warp_sum(b);
+    c = warp_sum(c);
+    if ((tid & 31) == 0) { wsum[0][tid >> 5] = a; wsum[1][tid >> 5] = b; wsum[2][tid >> 5] = c; }
     __syncthreads();
-    if (tid < n) {
-        double x = 0.0, y = 0.0;
-        for (int q = 0; q < groups; ++q) {
-            const double2 p = red[q * jp + tid];
-            x += p.x;
-            y += p.y;
-        }
-        e_out[tid] = make_double2(x, y);
+    if (tid == 0) {
+        double x = 0.0, y = 0.0, z = 0.0;
+        for (int w = 0; w < kReduceThreads / 32; ++w) { x += wsum[0][w]; y += wsum[1][w]; z += wsum[2][w]; }
+        record[2 * j] = x;
+        record[2 * j + 1] = y;
+        record[2 * n + j] = z;
     }
-    __syncthreads();
-}
-
-__global__ void __launch_bounds__(1024)
-cyc_project_finish_kernel(const double2* __restrict__ partial, int grid, int n, double2* e) {
-    __shared__ double2 red[1024];
-    block_sum_partials(partial, grid, n, red, e);
 }
 
 // The small solves below run either on the whole block (WARP = false: block-wide barriers, any size) or on its
@@ -592,34 +576,31 @@ constexpr int kSmallDim = 16;         // systems up to this size are solved in s
 
 // ------------------------------------------------------------------ locator after the projection
 __global__ void __launch_bounds__(kSolveThreads)
-cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ partial, int grid, const double2* __restrict__ e_in,
-                 int n, int s, double theta, uint8_t* flags, uint8_t* flags2, DeviceInfo* info) {
+cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, int n, int s, double theta, uint8_t* flags,
+                 uint8_t* flags2, DeviceInfo* info) {
     __shared__ double2 e[kMaxN], h[kMaxN], tw[kMaxN];
-    __shared__ double2 red[kSolveThreads];
     __shared__ double2 As[kSmallDim * kSmallDim], Vs[kSmallDim * kSmallDim];
     __shared__ double2 rhs_s[kMaxN / 2], beta_s[kMaxN / 2], coef_s[kMaxN / 2];
-    __shared__ double mag[kMaxN], sorted[kMaxN];
+    __shared__ double mag[kMaxN], sorted[kMaxN], qv[kMaxN];
     __shared__ int sh[4], count;
     __shared__ double scale_s, maxsyn_s;
     const int tid = threadIdx.x;
     const double rsn = 1.0 / sqrt((double)n);
 
-    if (tid < n) tw[tid] = cd->twiddle[tid];
-    if (e_in == nullptr) {
-        block_sum_partials(partial, grid, n, red, e);
-    } else {
-        if (tid < n) e[tid] = e_in[tid];
-        __syncthreads();
+    if (tid < n) {                                         // the projection record: n (re, im) pairs, then n values q_j
+        tw[tid] = cd->twiddle[tid];
+        e[tid] = e_in[tid];
+        qv[tid] = reinterpret_cast<const double*>(e_in + n)[tid];
     }
+    __syncthreads();
     if (tid < n) {
-        const double2 v = e[tid];
-        cd->e[tid] = v;
-        mag[tid] = sqrt(cabs2(v));
+        cd->e[tid] = e[tid];
+        mag[tid] = sqrt(qv[tid]);
         h[tid] = make_double2(0.0, 0.0);
     }
     if (tid == 0) count = 0;
     __syncthreads();
-    // median of |e_j| by rank counting
+    // scale = median of q_j^(1/2) by rank counting
     if (tid < n) {
         int rank = 0;
         for (int k = 0; k < n; ++k) rank += (mag[k] < mag[tid]) || (mag[k] == mag[tid] && k < tid);
@@ -839,55 +820,59 @@ cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n
 
 }  // namespace
 
-// Blocks of the projection: four per SM (six measured slower at n = 15); three per SM is what the
-// shared-memory sums of the n > 64 kernel allow.
-int project_grid_size(int sm_count, int n) { return sm_count * (n <= 64 ? 4 : 3); }
+// Blocks of the projection: four per SM (six measured slower at n = 15).
+int project_grid_size(int sm_count, int) { return sm_count * 4; }
 int project_grid_size(int sm_count) { return sm_count * 4; }
+
+// All launches of one projection: n <= 16 the few-rows kernel, n <= 64 one launch of the tile kernel, otherwise two
+// launches of it over half the rows each.  partial: [grid][n] double2 followed by [grid][n] double.
+static cudaError_t launch_project_kernels(int grid, cudaStream_t st, const float2* R, const float* f, int64_t len,
+                                          int64_t ld, int n, double2* partial, int accumulate) {
+    const bool vec2 = (ld % 2 == 0);
+    if (n <= 16) {
+        if (vec2) cyc_project_fewrows_kernel<true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, partial, accumulate);
+        else cyc_project_fewrows_kernel<false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, partial, accumulate);
+        return cudaGetLastError();
+    }
+    const int parts = n <= 64 ? 1 : 2;
+    const int per = (n + parts - 1) / parts;
+    for (int row0 = 0; row0 < n; row0 += per) {
+        const int nrows = (n - row0) < per ? (n - row0) : per;
+        if (nrows <= 32) {
+            if (vec2) cyc_project_kernel<4, true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, accumulate);
+            else cyc_project_kernel<4, false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, accumulate);
+        } else {
+            if (vec2) cyc_project_kernel<8, true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, accumulate);
+            else cyc_project_kernel<8, false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, accumulate);
+        }
+        const cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+    }
+    return cudaSuccess;
+}
 
 int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t len, int64_t ld, bool accumulate,
                        cudaStream_t st) {
-    const int grid = p->project_grid;
-    const bool vec2 = (ld % 2 == 0);
-    const int n = p->n;
-#define DRACO_PROJ(RPW, V2) \
-    cyc_project_kernel<RPW, V2><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0)
-    if (n > 64) {
-        const size_t smem = sizeof(float) * kProjectTile + sizeof(double2) * kThreads * ((n + kProjectWarps - 1) / kProjectWarps);
-        static bool configured_dev[64] = {};
-        bool& configured = configured_dev[(p->device >= 0 && p->device < 64) ? p->device : 0];
-        if (!configured) {
-            DRACO_CUDA(cudaFuncSetAttribute(cyc_project_manyrows_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)(sizeof(float) * kProjectTile + sizeof(double2) * kThreads * 16)));
-            DRACO_CUDA(cudaFuncSetAttribute(cyc_project_manyrows_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)(sizeof(float) * kProjectTile + sizeof(double2) * kThreads * 16)));
-            configured = true;
-        }
-        if (vec2) cyc_project_manyrows_kernel<true><<<grid, kThreads, smem, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
-        else cyc_project_manyrows_kernel<false><<<grid, kThreads, smem, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
-    } else if (n <= 16) {
-        if (vec2) cyc_project_fewrows_kernel<true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
-        else cyc_project_fewrows_kernel<false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, p->partial_dev, accumulate ? 1 : 0);
-    } else if (vec2) {
-        if (n <= 32) DRACO_PROJ(4, true);
-        else DRACO_PROJ(8, true);
-    } else {
-        if (n <= 32) DRACO_PROJ(4, false);
-        else DRACO_PROJ(8, false);
-    }
-#undef DRACO_PROJ
-    DRACO_CUDA(cudaGetLastError());
+    DRACO_CUDA(launch_project_kernels(p->project_grid, st, R, f, len, ld, p->n, p->partial_dev, accumulate ? 1 : 0));
     return DRACO_OK;
 }
 
 int launch_cyc_project_finish(draco_plan* p, double2* e_out, cudaStream_t st) {
-    cyc_project_finish_kernel<<<1, 1024, 0, st>>>(p->partial_dev, p->project_grid, p->n, e_out);
+    cyc_reduce_partials_kernel<<<p->n, kReduceThreads, 0, st>>>(p->partial_dev, p->project_grid, p->n,
+                                                                reinterpret_cast<double*>(e_out));
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }
 
+// e == nullptr: the record of the plan's own projection (launch_cyc_project) is formed first
 int launch_cyc_solve(draco_plan* p, const double2* e, uint8_t* flags, cudaStream_t st) {
-    cyc_solve_kernel<<<1, kSolveThreads, 0, st>>>(p->cyc_dev, p->partial_dev, p->project_grid, e, p->n, p->s, p->theta,
-                                                  flags, p->flags_dev, p->info_dev);
+    if (!e) {
+        double2* own = reinterpret_cast<double2*>(p->cyc_dev->record);      // address arithmetic only: cyc_dev is a device pointer
+        const int rc = launch_cyc_project_finish(p, own, st);
+        if (rc != DRACO_OK) return rc;
+        e = own;
+    }
+    cyc_solve_kernel<<<1, kSolveThreads, 0, st>>>(p->cyc_dev, e, p->n, p->s, p->theta, flags, p->flags_dev, p->info_dev);
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }
@@ -906,11 +891,12 @@ int launch_cyc_decode_vector(draco_plan* p, const uint8_t* flags, cudaStream_t s
 // fails or fragments the pool), or a step loop that cannot afford the implicit device-wide
 // synchronisation an allocation or a free may cause.  For them the block partials of the
 // projection live in this fixed array instead of in a plan.  Every GPU that loads the library
-// carries its 592 KB until the process exits.
+// carries its 888 KB until the process exits.
 namespace draco {
 namespace {
 constexpr int kStaticGridMax = 296;                                   // blocks whose partials fit
-static __device__ __align__(256) double2 g_static_partial[kStaticGridMax * kMaxN];
+// per block and node one double2 (partial of e_j) and, after all of those, one double (partial of q_j)
+static __device__ __align__(256) double2 g_static_partial[kStaticGridMax * kMaxN * 3 / 2];
 constexpr int kMaxDevices = 64;
 double2* g_static_partial_ptr[kMaxDevices] = {};                      // device address per device, set once
 int g_static_sm_count[kMaxDevices] = {};
@@ -952,17 +938,8 @@ extern "C" int draco_cyc_project_noalloc(int n, int64_t d, const void* R, const 
     const float2* Rc = static_cast<const float2*>(R);
     // Every block writes its n partials (zeros if it had no tile), so nothing has to be cleared
     // between calls even though the array keeps the previous call's contents.
-    if (d % 2 == 0) {
-        if (n <= 32) cyc_project_kernel<4, true><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
-        else if (n <= 64) cyc_project_kernel<8, true><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
-        else cyc_project_kernel<16, true><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
-    } else {
-        if (n <= 32) cyc_project_kernel<4, false><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
-        else if (n <= 64) cyc_project_kernel<8, false><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
-        else cyc_project_kernel<16, false><<<grid, kThreads, 0, st>>>(Rc, f, d, d, n, partial, 0);
-    }
-    DRACO_CUDA(cudaGetLastError());
-    cyc_project_finish_kernel<<<1, 1024, 0, st>>>(partial, grid, n, reinterpret_cast<double2*>(e));
+    DRACO_CUDA(launch_project_kernels(grid, st, Rc, f, d, d, n, partial, 0));
+    cyc_reduce_partials_kernel<<<n, kReduceThreads, 0, st>>>(partial, grid, n, e);
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }

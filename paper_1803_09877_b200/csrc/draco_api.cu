@@ -176,8 +176,10 @@ int draco_plan_create(int n, int s, int64_t d, int code, draco_plan** out) {
         DRACO_TRY(cudaMemcpy(p->taps_full_dev, taps_full.data(), sizeof(float2) * taps_full.size(),
                              cudaMemcpyHostToDevice));
         p->project_grid = project_grid_size(p->sm_count, n);
-        DRACO_TRY(cudaMalloc(&p->partial_dev, sizeof(double2) * (size_t)p->project_grid * n));
-        DRACO_TRY(cudaMemset(p->partial_dev, 0, sizeof(double2) * (size_t)p->project_grid * n));
+        // per block and node: a double2 partial of e_j, then (after all of those) a double partial of q_j
+        const size_t partial_bytes = (sizeof(double2) + sizeof(double)) * (size_t)p->project_grid * n;
+        DRACO_TRY(cudaMalloc(&p->partial_dev, partial_bytes));
+        DRACO_TRY(cudaMemset(p->partial_dev, 0, partial_bytes));
     }
 #undef DRACO_TRY
     *out = p;

@@ -48,6 +48,7 @@ struct CycDevice {
     double2 work[kMaxN * (kMaxN + 1)];  // elimination work space
     double2 vec[4 * kMaxN];
     int32_t perm[kMaxN];
+    double record[3 * kMaxN];         // the plan's own projection record: n (re, im) pairs, then n values q_j
 };
 
 struct DeviceInfo {                   // mirrors draco_info

@@ -2,9 +2,10 @@
 
 Every step of the path is independent per coordinate except the locator's
 projection e = f R, a sum over coordinates.  So rank p keeps columns
-[c0, c1) of all n rows, and the only exchange is one all-reduce of the n complex
-projections (2 n doubles) between the projection kernel and the small locator
-solve, which every rank then repeats identically.  The repetition code needs no
+[c0, c1) of all n rows, and the only exchange is one all-reduce of the projection
+record (3 n doubles: the n complex projections and the n squared vector norms that
+set the locator's rank cutoff; both add up over coordinates) between the projection
+kernel and the small locator solve, which every rank then repeats identically.  The repetition code needs no
 exchange for the sum; its per-node flags are OR-ed (a MAX all-reduce of n bytes).
 """
 from __future__ import annotations
@@ -25,7 +26,7 @@ def shard_range(d_total: int, world: int, rank: int, align: int = 2048) -> tuple
 def locate_sharded(plan, R, f, flags, e_buf, group=None, stream=None):
     """Cyclic locator over a d-sharded R: local projection, all-reduce(sum) of e, local solve.
 
-    ``plan`` is the rank's plan for its own slice; ``e_buf`` a float64 tensor of 2 n
+    ``plan`` is the rank's plan for its own slice; ``e_buf`` a float64 tensor of 3 n
     values on the same device as R.  Every rank ends with the same flags.
     """
     import torch.distributed as dist

@@ -71,10 +71,12 @@ def test_locate_and_decode_parity_on_identical_R(n, s, d, n_adv_mode):
     want = orc.cyc_locate(R, f, n, s)
     Rd, fd = dev(R), dev(f)
     # projection
-    e = torch.empty(2 * n, dtype=torch.float64, device="cuda")
+    e = torch.empty(3 * n, dtype=torch.float64, device="cuda")        # n (re, im) pairs, then n squared norms q_j
     plan.cyc_project(Rd, fd, e)
-    eg = host(e).view(np.complex128)
+    eg = host(e)[: 2 * n].view(np.complex128)
     assert np.abs(eg - want["e"]).max() <= 1e-6 * np.abs(want["e"]).max()
+    qo = orc.cyc_project_energy(R)
+    assert np.abs(host(e)[2 * n:] - qo).max() <= 1e-5 * qo.max()      # fp32 terms: a yardstick, not a result
     # locator
     flags = torch.full((n,), 9, dtype=torch.uint8, device="cuda")
     plan.locate(Rd, fd, flags)
@@ -87,7 +89,7 @@ def test_locate_and_decode_parity_on_identical_R(n, s, d, n_adv_mode):
     np.testing.assert_array_equal(fg, want["flags"])
     assert sorted(np.flatnonzero(fg)) == adv.tolist()
     assert info["locator_rank"] == want["rank"] == n_adv and info["n_flagged"] == n_adv
-    assert abs(info["scale"] - want["scale"]) <= 1e-6 * want["scale"]
+    assert abs(info["scale"] - want["scale"]) <= 1e-5 * want["scale"]
     # split entry points agree with the fused one
     flags2 = torch.empty_like(flags)
     plan.cyc_locate_from_projection(e, flags2)
@@ -248,9 +250,9 @@ def test_full_size_resnet152_config_sampled():
     err = normwise(host(u[idx]), exact)
     assert err <= 2.0 * floor + 1e-6, (err, floor)
     # projection of two honest rows over all d, by the oracle's definition in chunks
-    e = torch.empty(2 * n, dtype=torch.float64, device="cuda")
+    e = torch.empty(3 * n, dtype=torch.float64, device="cuda")
     plan.cyc_project(Z, f, e)
-    eg = host(e).view(np.complex128)
+    eg = host(e)[: 2 * n].view(np.complex128)
     W = orc.cyc_W(n, s)
     for j in (int(honest[0]), int(honest[-1])):
         acc = 0.0 + 0.0j

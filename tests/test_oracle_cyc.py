@@ -255,3 +255,32 @@ def test_packed_pipeline_corrects_every_placement(n, s, d):
             u = orc.cyc_decode_packed(R, n, s, loc["flags"], d)
             assert u.shape == (d,)
             assert np.abs(u - exact).max() <= 1e-8 * np.abs(exact).max()
+
+
+def test_rank_cutoff_is_measured_against_the_size_of_the_vectors_not_of_their_projection():
+    """r = n (one row in C_L): every honest node sends the same vector, so all e_j coincide and, for an f that makes
+    that one signed sum cancel, median_j |e_j| is tiny while the rounding noise of the vectors is not.  The cutoff
+    theta * median_j q_j^(1/2) must still call rounding-level differences between the rows rank 0, and must still
+    see real adversaries."""
+    n, s, d = 15, 7, 4096
+    G = di.gradient_rows(31, n, d)
+    Z = orc.cyc_encode(G, n, s)
+    rng = np.random.default_rng(5)
+    f = di.projection_vector(32, d).astype(np.float64)
+    f -= (Z[0].real @ f) / (Z[0].real @ Z[0].real) * Z[0].real * (1 - 1e-3)         # e_j shrinks to 1e-3 of its size
+    noisy = (Z * (1 + 2.0 ** -24 * rng.uniform(-1, 1, Z.shape))).astype(np.complex64)   # rows differ by fp32 rounding
+    e, q = orc.cyc_project(noisy, f), orc.cyc_project_energy(noisy)
+    assert np.median(np.abs(e)) < 0.02 * np.median(np.sqrt(q))                      # the sum did cancel
+    loc = orc.cyc_locate(noisy, f, n, s)
+    assert loc["rank"] == 0 and not loc["flags"].any()
+    assert abs(loc["scale"] - np.median(np.sqrt(q))) <= 1e-12 * loc["scale"]
+    # against |e_j| the same rows look like seven adversaries
+    assert orc.cyc_locate_from_projection(e, np.abs(e) ** 2, n, s)["rank"] > 0
+    # q by its definition, term by term
+    j = 3
+    assert abs(q[j] - sum(abs(complex(noisy[j, i])) ** 2 for i in range(d))) <= 1e-10 * q[j]
+    adv = [2, 9, 13]
+    R = noisy.copy()
+    R[adv] *= -100
+    loc = orc.cyc_locate(R, di.projection_vector(33, d), n, s)
+    assert sorted(np.flatnonzero(loc["flags"])) == adv

@@ -32,11 +32,13 @@ class _OraclePlan:
         self.n, self.s = n, s
 
     def cyc_project(self, R, f, e, stream=None):
-        val = orc.cyc_project(R.numpy().view(np.complex64), f.numpy())
-        e.copy_(torch.from_numpy(val.view(np.float64)))
+        Rc = R.numpy().view(np.complex64)
+        val = orc.cyc_project(Rc, f.numpy())
+        e[: 2 * self.n].copy_(torch.from_numpy(val.view(np.float64)))
+        e[2 * self.n:].copy_(torch.from_numpy(orc.cyc_project_energy(Rc)))
 
     def cyc_locate_from_projection(self, e, flags, stream=None):
-        out = orc.cyc_locate_from_projection(e.numpy().view(np.complex128), self.n, self.s)
+        out = orc.cyc_locate_from_projection(e.numpy()[: 2 * self.n].view(np.complex128), e.numpy()[2 * self.n:], self.n, self.s)
         flags.copy_(torch.from_numpy(out["flags"].astype(np.uint8)))
 
 
@@ -51,7 +53,7 @@ def _worker(rank, world, port, n, s, d, adv, result):
     di.apply_adversaries(R, adv, [di.ADV_REVGRAD] * len(adv), [100.0] * len(adv), seed=9, i0=c0)
     f = di.projection_vector(8, d, i0=c0, i1=c1)
     flags = torch.zeros(n, dtype=torch.uint8)
-    e = torch.zeros(2 * n, dtype=torch.float64)
+    e = torch.zeros(3 * n, dtype=torch.float64)
     locate_sharded(_OraclePlan(n, s), torch.from_numpy(R.view(np.float32)), torch.from_numpy(f), flags, e)
     u = orc.cyc_decode(R, n, s, flags.numpy().astype(bool))
     rep_flags = torch.zeros(n, dtype=torch.uint8)
@@ -79,7 +81,8 @@ def test_two_rank_sharded_locate_and_decode():
     for r in range(world):
         flags, e, u, (c0, c1), rep_flags = result[r]
         assert sorted(np.flatnonzero(flags)) == adv
-        np.testing.assert_allclose(e.view(np.complex128), whole["e"], rtol=1e-10, atol=1e-6 * whole["scale"])
+        np.testing.assert_allclose(e[: 2 * n].view(np.complex128), whole["e"], rtol=1e-10, atol=1e-6 * whole["scale"])
+        np.testing.assert_allclose(e[2 * n:], orc.cyc_project_energy(R), rtol=1e-10)
         exact = G[:, c0:c1].astype(np.float64).sum(axis=0)
         assert np.abs(u - exact).max() <= 1e-4 * np.abs(exact).max()
         assert rep_flags.tolist()[:2] == [1, 1] and rep_flags.sum() == 2

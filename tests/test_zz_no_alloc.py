@@ -20,21 +20,24 @@ def _project_both_ways(dr, n, s, d, seed):
     R = torch.from_numpy(di.complex_rows(seed, n, d, std=3.0).view(np.float32)).cuda()
     f = torch.from_numpy(di.projection_vector(seed + 1, d)).cuda()
     plan = dr.Plan(n, s, d, dr.CYC)
-    e_plan = torch.zeros(2 * n, dtype=torch.float64, device="cuda")
+    e_plan = torch.zeros(3 * n, dtype=torch.float64, device="cuda")          # n (re, im) pairs, then n squared norms q_j
     plan.cyc_project(R, f, e_plan)
-    e_static = torch.full((2 * n,), float("nan"), dtype=torch.float64, device="cuda")
+    e_static = torch.full((3 * n,), float("nan"), dtype=torch.float64, device="cuda")
     dr.cyc_project_noalloc(n, d, R, f, e_static)
     torch.cuda.synchronize()
-    return e_plan.cpu().numpy().view(np.complex128), e_static.cpu().numpy().view(np.complex128)
+    return e_plan.cpu().numpy(), e_static.cpu().numpy()
 
 
 def test_noalloc_projection_matches_plan_projection_twice_in_a_row():
     import paper_1803_09877_b200 as dr
     for call, (n, s, d) in enumerate([(45, 5, 300_004), (15, 2, 4099)]):     # vector path, then the odd-d scalar path
         want, got = _project_both_ways(dr, n, s, d, seed=100 + call)
-        assert np.all(np.isfinite(got.view(np.float64)))
-        assert np.abs(got - want).max() <= 1e-6 * np.abs(want).max()           # tolerance of the projection parity tests
-        assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()          # same kernel; only the number of block partials differs
+        assert np.all(np.isfinite(got))
+        we, ge = want[: 2 * n].view(np.complex128), got[: 2 * n].view(np.complex128)
+        assert np.abs(ge - we).max() <= 1e-6 * np.abs(we).max()                # tolerance of the projection parity tests
+        assert np.abs(ge - we).max() <= 1e-12 * np.abs(we).max()               # same kernel; only the number of block partials differs
+        # the squared norms are a yardstick (few-row plans add their fp32 terms in fp32): a few digits
+        assert np.abs(got[2 * n:] - want[2 * n:]).max() <= 1e-5 * want[2 * n:].max() and want[2 * n:].min() > 0
 
 
 def test_noalloc_projection_rejects_sizes_beyond_its_fixed_capacity():
