@@ -332,7 +332,9 @@ def run_gpu(args):
                           "frac_of_nominal_8TBps": round(g / 8000.0, 4)}
         else:
             stages[nm] = {"ms": round(stage_ms[nm], 4)}
-    launches = (1 + len(adv) + (2 if cyc else 0) + 2 + (1 if (cyc and world > 1) else 0)) * args.steps
+    # encode 1, corrupt 1 per adversary, cyclic locate = projection (two launches over half the rows each when n > 64)
+    # + reduction of the block partials + solve, decode = decode vector + recovery (repetition: vote + finish)
+    launches = (1 + len(adv) + ((3 + (1 if n > 64 else 0)) if cyc else 0) + 2) * args.steps
 
     # the same step captured once into a CUDA graph and replayed (one GPU only: the sharded step has a collective)
     graph_replay = None
