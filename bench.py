@@ -523,6 +523,24 @@ def run_sweep(args):
                "min_encode_frac_large_d": min((x["encode_frac"] for x in big), default=None), "out": args.sweep_out}
     print(json.dumps(summary))
 
+def sweep_table(path: str) -> str:
+    """Markdown table of a finished sweep (the JSON lines that --sweep wrote)."""
+    rows = [json.loads(l) for l in open(path) if l.strip()]
+    rows = [r for r in rows if "n" in r and "encode_ms" in r]
+    def dfmt(d):
+        return f"{d / 1e6:.1f} M"
+    out = ["| code | n | s | d | encode ms | encode GB/s (frac) | locate+decode ms | decode GB/s (frac) | coded GB/s produced / consumed "
+           "| err 0 adv | err s adv | flags ≤ s | > s fails |", "|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
+    for r in rows:
+        c = r["checks"]
+        out.append(f"| {r['code']} | {r['n']} | {r['s']} | {dfmt(r['d'])} | {r['encode_ms']:.3f} | {r['encode_hbm_GBps']:.0f} ({r['encode_frac']:.2f}) "
+                   f"| {r['decode_ms']:.3f} | {r['decode_hbm_GBps']:.0f} ({r['decode_frac']:.2f}) "
+                   f"| {r['coded_GBps_produced']:.0f} / {r['coded_GBps_consumed']:.0f} | {c['0']['err']:.1e} | {c['s']['err']:.1e} "
+                   f"| {'yes' if r['flags_ok_upto_s'] else 'NO'} | {'yes' if r['beyond_s_fails'] else 'NO'} |")
+    return "\n".join(out) + "\n"
+
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -537,10 +555,14 @@ def main():
     ap.add_argument("--sweep-n", default="15,45,105")
     ap.add_argument("--sweep-s", default="1,2,5,7")
     ap.add_argument("--sweep-d", default="1e6,11.7e6,60.2e6,138e6")
+    ap.add_argument("--sweep-table", default=None, help="render the JSON lines of a finished sweep as a markdown table on stdout (no GPU)")
     ap.add_argument("--sweep-out", default=os.path.join(ROOT, "gpurun_out", "sweep.jsonl"))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.sweep_table:
+        sys.stdout.write(sweep_table(args.sweep_table))
+        return
     if args.d is not None:
         w = list(WORKLOADS[args.workload])
         w[3] = args.d

@@ -645,12 +645,23 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, int n, int s, 
         }
         if (tid < s) rhs_s[tid] = h[n - 1 - tid];
         __syncthreads();
-        if (small) {
-            if (tid < 32) warp_jacobi_pinv(A, V, rhs_s, s, tol, beta_s, coef_s, sh);
-            __syncthreads();
-            rank = sh[1];
-        } else {
-            rank = block_jacobi_pinv(A, V, rhs_s, s, tol, beta_s, coef_s, sh);
+        // No singular value exceeds the Frobenius norm: when that is within the cutoff (the usual step without any
+        // adversary, where the syndromes are rounding noise) the rank is 0 and the SVD is skipped.
+        if (tid < 32) {
+            double fro2 = 0.0;
+            for (int idx = tid; idx < sp * sp; idx += 32) fro2 += cabs2(A[idx]);
+            fro2 = warp_sum(fro2);
+            if (tid == 0) sh[2] = (fro2 > tol * tol) ? 1 : 0;
+        }
+        __syncthreads();
+        if (sh[2]) {
+            if (small) {
+                if (tid < 32) warp_jacobi_pinv(A, V, rhs_s, s, tol, beta_s, coef_s, sh);
+                __syncthreads();
+                rank = sh[1];
+            } else {
+                rank = block_jacobi_pinv(A, V, rhs_s, s, tol, beta_s, coef_s, sh);
+            }
         }
     }
     if (rank > 0) {
