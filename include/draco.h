@@ -76,6 +76,14 @@ typedef struct draco_info {
     int32_t internal_error; /* non-zero: a kernel gave up a bounded wait (sticky); draco_get_info then returns DRACO_EINTERNAL.
                                Always 0 with the current kernels, none of which spins on a flag */
     int32_t reserved;
+    double locator_margin; /* cyclic locate: |t| of the weakest flagged node / |t| of the strongest unflagged one (exactly
+                              `rank` entries of t are non-zero in exact arithmetic, so this is large when the flags can be
+                              trusted and near 1 when they cannot); 1e300 when no node or every node is flagged */
+    double im_residual;    /* cyclic decode, unpacked plans: max |Im(u-hat_i)| over the coordinates i with floor(i / 64) mod 8 = 0.
+                              u-hat = R_{.,U} b is real when every node of U is honest, so against re_max this tells a decode
+                              whose U still holds an adversary (wrong or missing flags, more than s adversaries) from a good
+                              one, whose residual is the rounding floor of complex64 vectors; 0 for packed plans */
+    double re_max;         /* the same maximum of |Re(u-hat_i)|, the scale for im_residual */
 } draco_info;
 
 /*

@@ -24,7 +24,8 @@ class DracoError(RuntimeError):
 class DracoInfo(C.Structure):
     _fields_ = [("status", C.c_int32), ("n_flagged", C.c_int32), ("locator_rank", C.c_int32),
                 ("n_active", C.c_int32), ("no_majority", C.c_uint64), ("scale", C.c_double),
-                ("max_syndrome", C.c_double), ("internal_error", C.c_int32), ("reserved", C.c_int32)]
+                ("max_syndrome", C.c_double), ("internal_error", C.c_int32), ("reserved", C.c_int32),
+                ("locator_margin", C.c_double), ("im_residual", C.c_double), ("re_max", C.c_double)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}

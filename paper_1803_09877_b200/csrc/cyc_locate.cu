@@ -1,6 +1,8 @@
 // Cyclic-code adversary locator phi(R) (Section 3, "Cyclic Code"; correctness: Lemmas 4, 6-8).
 //
-//   cyc_project_kernel   e_j = sum_i f_i R[j][i]: the one O(d P) step, a single pass over R.
+//   cyc_project_kernel   e_j = sum_i f_i R[j][i]: the one O(d P) step, a single pass over R; beside it
+//                        q_j = sum_i |R[j][i]|^2, the yardstick of the rank cutoff below.
+//   cyc_reduce_partials_kernel   the blocks' partial sums of e and q added up in a fixed order.
 //   cyc_solve_kernel     [h_{n-2s} .. h_{n-1}] = e C_R^dagger, the s x s Toeplitz system for
 //                        beta (pseudo-inverse by a Jacobi SVD: its rank = the number of
 //                        adversaries seen), the recurrence h_l = sum_u beta_u h_{l+u-s}, t = C h,
@@ -699,6 +701,8 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, int n, int s, 
             int pos = 0;
             for (int k = 0; k < n; ++k) pos += (mag[k] > mag[tid]) || (mag[k] == mag[tid] && k < tid);
             flagged = pos < rank;
+            if (pos == rank - 1) sorted[0] = mag[tid];     // |t|^2 of the weakest flagged node ..
+            if (pos == rank) sorted[1] = mag[tid];         // .. and of the strongest unflagged one
         }
     } else if (tid < n) {
         cd->t[tid] = make_double2(0.0, 0.0);
@@ -717,6 +721,7 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, int n, int s, 
         info->max_syndrome = maxsyn_s;
         info->status = DRACO_OK;
         info->no_majority = 0;
+        info->locator_margin = (rank > 0 && rank < n) ? sqrt(sorted[0] / fmax(sorted[1], 1e-300)) : 1e300;
     }
 }
 
@@ -749,7 +754,10 @@ cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n
     const int a = a_s;
     if (a > 2 * s) {                                       // fewer than n - 2 s rows left: no b exists
         if (tid < n) cd->b[tid] = make_double2(0.0, 0.0);
-        if (tid == 0) { info->n_active = 0; info->n_flagged = a; info->status = DRACO_ETOOMANY; }
+        if (tid == 0) {
+            info->n_active = 0; info->n_flagged = a; info->status = DRACO_ETOOMANY;
+            info->im_residual_bits = 0ull; info->re_max_bits = 0ull;
+        }
         return;
     }
     double2* x = x_s;
@@ -825,6 +833,8 @@ cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n
     if (tid == 0) {
         info->n_active = n - a;
         info->n_flagged = a;
+        info->im_residual_bits = 0ull;                     // the recovery kernel's blocks merge their maxima into these
+        info->re_max_bits = 0ull;
         if (info->status == DRACO_ETOOMANY) info->status = DRACO_OK;
     }
 }

@@ -4,6 +4,11 @@
 // One pass over the rows with b_j != 0.  The code cancels entries of W as large as 1e5 back
 // to 1, so the running sums are kept in fp64 (fp32 would lose about kappa * 2^-24 of the
 // result); R stays fp32 in memory.  HBM traffic: 8 |U| len bytes read + 4 len written.
+//
+// Self-check (unpacked plans).  u-hat = G 1_P is real, so Im(u-hat) is rounding residue as long as every
+// row of U is honest, and of the size of the result when an adversary is left in U.  The kernel forms
+// Im(u-hat_i) on one coordinate run in eight (floor(i / 64) mod 8 = 0: a warp-uniform choice, 12 % more
+// arithmetic) and leaves max |Im| and max |Re| over those coordinates in the plan's info block.
 #include "draco_internal.cuh"
 
 namespace draco {
@@ -18,11 +23,11 @@ constexpr int kUnroll = 8;
 template <bool VEC2, bool PACKED>
 __global__ void __launch_bounds__(kThreads)
 cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const CycDevice* __restrict__ cd,
-                   const DeviceInfo* __restrict__ info, float* __restrict__ u, int64_t d_packed, float* __restrict__ w,
-                   float scale) {
+                   DeviceInfo* info, float* __restrict__ u, int64_t d_packed, float* __restrict__ w, float scale) {
     __shared__ double2 bs[kMaxN];
     __shared__ int rows[kMaxN];
     const int count = info->n_active;
+    double im_max = 0.0, re_max = 0.0;                    // over this thread's sampled coordinates
     for (int k = threadIdx.x; k < count; k += kThreads) {
         bs[k] = cd->b_active[k];
         rows[k] = cd->active[k];
@@ -33,6 +38,7 @@ cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const 
         const int64_t nvec = len / 2;
         for (int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x; v < nvec; v += stride) {
             const float2* col = R + v * 2;
+            const bool sampled = !PACKED && ((v >> 5) & 7) == 0;       // coordinates 2 v, 2 v + 1: floor(i / 64) mod 8 == 0
             double a0 = 0.0, a1 = 0.0, i0 = 0.0, i1 = 0.0;
             for (int k0 = 0; k0 < count; k0 += kUnroll) {
                 float4 x[kUnroll];
@@ -48,13 +54,17 @@ cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const 
                         a0 = fma(-b.y, xi0, a0);
                         a1 = fma(b.x, xr1, a1);
                         a1 = fma(-b.y, xi1, a1);
-                        if (PACKED) {
+                        if (PACKED || sampled) {
                             i0 = fma(b.x, xi0, i0);
                             i0 = fma(b.y, xr0, i0);
                             i1 = fma(b.x, xi1, i1);
                             i1 = fma(b.y, xr1, i1);
                         }
                     }
+            }
+            if (sampled) {
+                im_max = fmax(im_max, fmax(fabs(i0), fabs(i1)));
+                re_max = fmax(re_max, fmax(fabs(a0), fabs(a1)));
             }
             if (u != nullptr) {
                 __stcs(reinterpret_cast<float2*>(u + v * 2), make_float2((float)a0, (float)a1));
@@ -77,16 +87,21 @@ cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const 
         }
     } else {
         for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < len; i += stride) {
+            const bool sampled = !PACKED && ((i >> 6) & 7) == 0;
             double a0 = 0.0, i0 = 0.0;
             for (int k = 0; k < count; ++k) {
                 const float2 x = __ldcs(R + (int64_t)rows[k] * ld + i);
                 const double2 b = bs[k];
                 a0 = fma(b.x, (double)x.x, a0);
                 a0 = fma(-b.y, (double)x.y, a0);
-                if (PACKED) {
+                if (PACKED || sampled) {
                     i0 = fma(b.x, (double)x.y, i0);
                     i0 = fma(b.y, (double)x.x, i0);
                 }
+            }
+            if (sampled) {
+                im_max = fmax(im_max, fabs(i0));
+                re_max = fmax(re_max, fabs(a0));
             }
             if (u != nullptr) {
                 u[i] = (float)a0;
@@ -96,6 +111,20 @@ cyc_recover_kernel(const float2* __restrict__ R, int64_t len, int64_t ld, const 
                 w[i] = fmaf(-scale, (float)a0, w[i]);
                 if (PACKED && len + i < d_packed) w[len + i] = fmaf(-scale, (float)i0, w[len + i]);
             }
+        }
+    }
+    if (!PACKED) {
+        // non-negative doubles order like their bit patterns; NaN (an adversary may send it) counts as the largest
+        if (!(im_max == im_max)) im_max = __longlong_as_double(0x7ff0000000000000ll);
+        if (!(re_max == re_max)) re_max = __longlong_as_double(0x7ff0000000000000ll);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            im_max = fmax(im_max, __shfl_xor_sync(0xffffffffu, im_max, off));
+            re_max = fmax(re_max, __shfl_xor_sync(0xffffffffu, re_max, off));
+        }
+        if ((threadIdx.x & 31) == 0) {
+            if (im_max > 0.0) atomicMax(&info->im_residual_bits, (unsigned long long)__double_as_longlong(im_max));
+            if (re_max > 0.0) atomicMax(&info->re_max_bits, (unsigned long long)__double_as_longlong(re_max));
         }
     }
 }

@@ -311,6 +311,9 @@ int draco_get_info(draco_plan* plan, draco_info* info, void* stream) {
     info->max_syndrome = h.max_syndrome;
     info->internal_error = h.internal_error;
     info->reserved = 0;
+    info->locator_margin = h.locator_margin;
+    memcpy(&info->im_residual, &h.im_residual_bits, sizeof(double));
+    memcpy(&info->re_max, &h.re_max_bits, sizeof(double));
     return h.internal_error ? DRACO_EINTERNAL : DRACO_OK;
 }
 

@@ -61,6 +61,9 @@ struct DeviceInfo {                   // mirrors draco_info
     double max_syndrome;
     int32_t internal_error;
     int32_t reserved;
+    double locator_margin;
+    unsigned long long im_residual_bits;   // bit patterns of non-negative doubles: they order like integers, so the
+    unsigned long long re_max_bits;        // blocks of the recovery kernel merge their maxima with atomicMax
 };
 
 }  // namespace draco

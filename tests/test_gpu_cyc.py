@@ -90,6 +90,13 @@ def test_locate_and_decode_parity_on_identical_R(n, s, d, n_adv_mode):
     assert sorted(np.flatnonzero(fg)) == adv.tolist()
     assert info["locator_rank"] == want["rank"] == n_adv and info["n_flagged"] == n_adv
     assert abs(info["scale"] - want["scale"]) <= 1e-5 * want["scale"]
+    # |t| of the weakest flagged node over |t| of the strongest unflagged one
+    if 0 < want["rank"] < n:
+        assert info["locator_margin"] > 10
+        # the denominator is the noise left on an honest node: the same order of magnitude on both sides, no more
+        assert 0.1 < info["locator_margin"] / want["margin"] < 10 or min(info["locator_margin"], want["margin"]) > 1e6
+    else:
+        assert info["locator_margin"] == 1e300
     # split entry points agree with the fused one
     flags2 = torch.empty_like(flags)
     plan.cyc_locate_from_projection(e, flags2)
@@ -106,6 +113,13 @@ def test_locate_and_decode_parity_on_identical_R(n, s, d, n_adv_mode):
     uo = orc.cyc_decode(R, n, s, want["flags"])
     assert normwise(host(u), uo) <= 1e-4
     assert normwise(host(u), uo) <= 1e-6                    # what fp64 accumulation actually delivers
+    # the decoder's self-check: Im(u-hat) on one 64-coordinate run in eight, against the oracle's u-hat there
+    uhat = orc.cyc_recover(R, bo)
+    sampled = (np.arange(d) // 64) % 8 == 0
+    im_o, re_o = np.abs(uhat.imag[sampled]).max(), np.abs(uhat.real[sampled]).max()
+    assert abs(info["re_max"] - re_o) <= 1e-6 * re_o
+    assert abs(info["im_residual"] - im_o) <= 1e-3 * im_o + 1e-12 * re_o
+    assert info["im_residual"] <= 1e-2 * info["re_max"]       # an honest U: rounding residue only
     u2 = torch.empty_like(u)
     f2 = torch.empty_like(flags)
     plan.locate_decode(Rd, fd, f2, u2)
@@ -181,6 +195,32 @@ def test_beyond_s_fails_visibly():
     wrong_set = sorted(np.flatnonzero(host(flags))) != adv
     wrong_sum = normwise(host(u), G.astype(np.float64).sum(axis=0)) > 1e-3
     assert wrong_set or wrong_sum or info["status"] != 0
+    # and the caller can see it without knowing the truth: an adversary left in U makes u-hat complex
+    assert info["im_residual"] > 0.1 * info["re_max"]
+
+
+def test_undetected_adversary_shows_in_the_self_checks():
+    """Six noise adversaries, three of them two nodes apart, at n = 44: the sixth singular value of the syndrome
+    system sinks below the rank cutoff of complex64 vectors, oracle and GPU both flag five nodes, and the sum is
+    wrong.  The margin between flagged and unflagged |t_j| and the imaginary residue of the decode both say so."""
+    n, s, d, seed = 44, 6, 257, 892766506
+    dr, plan = _plan(n, s, d)
+    G = di.gradient_rows(seed, n, d)
+    Z = torch.empty(n, 2 * d, dtype=torch.float32, device="cuda")
+    plan.encode(dev(G), Z)
+    adv = di.choose_adversaries(seed + 1, n, s)
+    plan.corrupt(Z, adv, [di.ADV_GAUSS] * s, [1e3] * s, seed=seed + 2)
+    f = di.projection_vector(seed + 3, d)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.locate_decode(Z, dev(f), flags, u)
+    info = plan.info()
+    want = orc.cyc_locate(host(Z).view(np.complex64), f, n, s)
+    np.testing.assert_array_equal(host(flags).astype(bool), want["flags"])
+    assert want["rank"] == s - 1 and sorted(np.flatnonzero(want["flags"])) != adv.tolist()
+    assert normwise(host(u), G.astype(np.float64).sum(axis=0)) > 1.0
+    assert info["locator_margin"] < 3 and want["margin"] < 3
+    assert info["im_residual"] > 0.1 * info["re_max"]
 
 
 def test_host_pipeline_matches_device_pipeline():
