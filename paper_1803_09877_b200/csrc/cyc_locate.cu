@@ -379,6 +379,22 @@ __device__ int block_gauss_jordan(double2* A, int dim, double tol, double2* x, i
     return rank;
 }
 
+// Rotation of one Jacobi pair from alpha = |a_p|^2, beta = |a_q|^2 and gamma = a_p^H a_q (g2 = |gamma|^2 > 0):
+// ph = exp(-i arg gamma), t = sign(zeta) / (|zeta| + sqrt(1 + zeta^2)) with zeta = (beta - alpha) / (2 |gamma|),
+// c = 1 / sqrt(1 + t^2), s = c t.  Written with four long-latency operations (two reciprocal square roots, a
+// square root and a division) instead of seven: t = sign(delta) 2 |gamma| / (|delta| + sqrt(delta^2 + 4 |gamma|^2)),
+// delta = beta - alpha.  The chain is serial and is most of a Jacobi step.
+__device__ __forceinline__ void jacobi_rotation(double alpha, double bet, double gr, double gi, double g2, double2& ph,
+                                                double& c, double& sn) {
+    const double rg = rsqrt(g2);
+    const double g = g2 * rg;
+    ph = make_double2(gr * rg, -gi * rg);
+    const double delta = bet - alpha;
+    const double tt = copysign(2.0 * g, delta) / (fabs(delta) + sqrt(fma(delta, delta, 4.0 * g2)));
+    c = rsqrt(fma(tt, tt, 1.0));
+    sn = c * tt;
+}
+
 // ------------------------------------------------------------------ small SVD solve
 // Pseudo-inverse solution of the s x s complex system A beta = rhs by one-sided (Hestenes)
 // Jacobi: columns of [A; V] are rotated in pairs until the columns of A are orthogonal; then
@@ -418,11 +434,9 @@ __device__ int block_jacobi_pinv(double2* A, double2* V, const double2* rhs, int
                 }
                 const double g2 = gr * gr + gi * gi;
                 if (g2 > 1e-30 * alpha * bet && g2 > 0.0) {
-                    const double g = sqrt(g2);
-                    const double2 ph = make_double2(gr / g, -gi / g);      // exp(-i arg gamma)
-                    const double zeta = (bet - alpha) / (2.0 * g);
-                    const double tt = copysign(1.0, zeta) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-                    const double c = 1.0 / sqrt(1.0 + tt * tt), sn = c * tt;
+                    double2 ph;
+                    double c, sn;
+                    jacobi_rotation(alpha, bet, gr, gi, g2, ph, c, sn);
                     for (int i = 0; i < s; ++i) {
                         const double2 x = ap[i], y = cmul(aq[i], ph);
                         ap[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
@@ -522,11 +536,9 @@ __device__ int warp_jacobi_pinv(double2* A, double2* V, const double2* rhs, int 
             }
             const double g2 = gr * gr + gi * gi;
             if (act && g2 > 1e-30 * alpha * bet && g2 > 0.0) {
-                const double g = sqrt(g2);
-                const double2 ph = make_double2(gr / g, -gi / g);      // exp(-i arg gamma)
-                const double zeta = (bet - alpha) / (2.0 * g);
-                const double tt = copysign(1.0, zeta) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-                const double c = 1.0 / sqrt(1.0 + tt * tt), sn = c * tt;
+                double2 ph;
+                double c, sn;
+                jacobi_rotation(alpha, bet, gr, gi, g2, ph, c, sn);
                 for (int i = sub; i < s; i += lp) {
                     const double2 x = ap[i], y = cmul(aq[i], ph);
                     ap[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
