@@ -1,0 +1,59 @@
+"""Cyclic code on many small random cases: shapes, adversary counts, attack models and seeds drawn from one seeded
+stream.  The GPU's flags must equal the oracle's on the very same received matrix in every case that does not sit on
+the rank cutoff, and where both find the planted adversaries the decoded sum must sit on the oracle's own complex64
+floor."""
+import numpy as np
+import pytest
+import torch
+
+import draco_inputs as di
+from oracle import draco_oracle as orc
+from gpu_util import dev, host, normwise
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("stream_seed", [11, 12])
+def test_random_small_cases_match_the_oracle(stream_seed):
+    import paper_1803_09877_b200 as dr
+    rng = np.random.default_rng(stream_seed)
+    both_found = on_the_edge = 0
+    for case in range(60):
+        n = int(rng.integers(3, 46))
+        s = int(rng.integers(1, min(7, (n - 1) // 2) + 1))
+        n_adv = int(rng.integers(0, s + 1))
+        d = int(rng.choice([257, 1000, 4096, 10001]))
+        model = int(rng.choice([di.ADV_REVGRAD, di.ADV_CONST, di.ADV_GAUSS]))
+        param = {di.ADV_REVGRAD: 100.0, di.ADV_CONST: 1e4, di.ADV_GAUSS: 1e3}[model]
+        seed = int(rng.integers(1, 1 << 30))
+        G = di.gradient_rows(seed, n, d)
+        f = di.projection_vector(seed + 3, d)
+        plan = dr.Plan(n, s, d, dr.CYC)
+        Z = torch.empty(n, 2 * d, dtype=torch.float32, device="cuda")
+        plan.encode(dev(G), Z)
+        adv = di.choose_adversaries(seed + 1, n, n_adv).tolist() if n_adv else []
+        if adv:
+            plan.corrupt(Z, adv, [model] * n_adv, [param] * n_adv, seed=seed + 2)
+        flags = torch.zeros(n, dtype=torch.uint8, device="cuda")
+        u = torch.zeros(d, dtype=torch.float32, device="cuda")
+        plan.locate_decode(Z, dev(f), flags, u)
+        info = plan.info()
+        R = host(Z).view(np.complex64)
+        want = orc.cyc_locate(R, f, n, s)
+        what = f"case {case}: n={n} s={s} adv={adv} model={model} d={d} seed={seed}"
+        tol = 1e-6 * want["scale"]
+        if any(tol / 3 < x < 3 * tol for x in want.get("sv", [])) or (0 < want["rank"] < n and want["margin"] < 10):
+            on_the_edge += 1         # a singular value at the rank cutoff, or |t| of flagged and unflagged nodes alike:
+            plan.close()             # rounding decides, and the two sides round differently
+            continue
+        np.testing.assert_array_equal(host(flags).astype(bool), want["flags"], err_msg=what)
+        assert info["locator_rank"] == want["rank"], what
+        if sorted(np.flatnonzero(want["flags"]).tolist()) == adv:
+            both_found += 1
+            exact = G.astype(np.float64).sum(axis=0)
+            floor = normwise(orc.cyc_decode(R, n, s, want["flags"]), exact)
+            assert normwise(host(u), exact) <= 2.0 * floor + 1e-6, what
+            assert info["im_residual"] <= 0.05 * info["re_max"], what
+        plan.close()
+    # the rest: clustered adversaries beyond what complex64 vectors can carry
+    assert on_the_edge <= 4 and both_found >= 54
