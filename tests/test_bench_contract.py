@@ -27,3 +27,18 @@ def test_non_zero_ranks_of_the_reference_arm_do_no_work():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0"],
                          capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_sweep_table_renders_one_row_per_point(tmp_path):
+    point = {"code": "cyc", "n": 15, "s": 2, "d": 1_000_000, "encode_ms": 0.05, "decode_ms": 0.08, "coded_GBps_produced": 2400.0,
+             "coded_GBps_consumed": 1500.0, "encode_hbm_GBps": 3600.0, "encode_frac": 0.55, "decode_hbm_GBps": 3000.0,
+             "decode_frac": 0.46, "checks": {"0": {"err": 2e-7}, "s": {"err": 3e-7}, ">s": {"err": 5.0}},
+             "flags_ok_upto_s": True, "beyond_s_fails": True}
+    path = tmp_path / "sweep.jsonl"
+    path.write_text(json.dumps(point) + "\n" + json.dumps(dict(point, n=45, flags_ok_upto_s=False)) + "\n" + json.dumps({"mode": "sweep"}) + "\n")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--sweep-table", str(path)], capture_output=True, text=True,
+                         timeout=120, cwd=ROOT)
+    assert out.returncode == 0, out.stderr
+    rows = [ln for ln in out.stdout.splitlines() if ln.startswith("| cyc")]
+    assert len(rows) == 2 and "| 15 | 2 | 1.0 M | 0.050 | 3600 (0.55) | 0.080 | 3000 (0.46) | 2400 / 1500 |" in rows[0]
+    assert rows[0].rstrip().endswith("| yes | yes |") and "| NO | yes |" in rows[1]
