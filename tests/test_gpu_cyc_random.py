@@ -57,3 +57,50 @@ def test_random_small_cases_match_the_oracle(stream_seed):
         plan.close()
     # the rest: clustered adversaries beyond what complex64 vectors can carry
     assert on_the_edge <= 4 and both_found >= 54
+
+
+def test_random_small_packed_cases_match_the_oracle():
+    """The same on the packed transport (Section 3, last paragraph): ceil(d / 2) complex entries per node, odd and
+    even d, the decoder returning [Re(u-hat); Im(u-hat)] cut to d entries."""
+    import paper_1803_09877_b200 as dr
+    rng = np.random.default_rng(31)
+    both_found = on_the_edge = 0
+    for case in range(60):
+        n = int(rng.integers(3, 46))
+        s = int(rng.integers(1, min(7, (n - 1) // 2) + 1))
+        n_adv = int(rng.integers(0, s + 1))
+        d = int(rng.choice([255, 1000, 4096, 8200, 10001]))
+        h = (d + 1) // 2
+        model = int(rng.choice([di.ADV_REVGRAD, di.ADV_CONST, di.ADV_GAUSS]))
+        param = {di.ADV_REVGRAD: 100.0, di.ADV_CONST: 1e4, di.ADV_GAUSS: 1e3}[model]
+        seed = int(rng.integers(1, 1 << 30))
+        G = di.gradient_rows(seed, n, d)
+        f = di.projection_vector(seed + 3, h)
+        plan = dr.Plan(n, s, d, dr.CYC_PACKED)
+        Z = torch.empty(n, 2 * h, dtype=torch.float32, device="cuda")
+        plan.encode(dev(G), Z)
+        adv = di.choose_adversaries(seed + 1, n, n_adv).tolist() if n_adv else []
+        if adv:
+            plan.corrupt(Z, adv, [model] * n_adv, [param] * n_adv, seed=seed + 2)
+        flags = torch.zeros(n, dtype=torch.uint8, device="cuda")
+        u = torch.zeros(d, dtype=torch.float32, device="cuda")
+        plan.locate_decode(Z, dev(f), flags, u)
+        info = plan.info()
+        R = host(Z).view(np.complex64)
+        want = orc.cyc_locate(R, f, n, s)
+        what = f"case {case}: n={n} s={s} adv={adv} model={model} d={d} seed={seed}"
+        tol = 1e-6 * want["scale"]
+        if any(tol / 3 < x < 3 * tol for x in want.get("sv", [])) or (0 < want["rank"] < n and want["margin"] < 10):
+            on_the_edge += 1
+            plan.close()
+            continue
+        np.testing.assert_array_equal(host(flags).astype(bool), want["flags"], err_msg=what)
+        assert info["locator_rank"] == want["rank"], what
+        if sorted(np.flatnonzero(want["flags"]).tolist()) == adv:
+            both_found += 1
+            uo = orc.cyc_decode_packed(R, n, s, want["flags"], d)
+            assert normwise(host(u), uo) <= 1e-6, what                   # identical R, identical flags
+            exact = G.astype(np.float64).sum(axis=0)
+            assert normwise(host(u), exact) <= 2.0 * normwise(uo, exact) + 1e-6, what
+        plan.close()
+    assert on_the_edge <= 4 and both_found >= 54
