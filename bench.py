@@ -556,7 +556,7 @@ def main():
     ap.add_argument("--sweep-s", default="1,2,5,7")
     ap.add_argument("--sweep-d", default="1e6,11.7e6,60.2e6,138e6")
     ap.add_argument("--sweep-table", default=None, help="render the JSON lines of a finished sweep as a markdown table on stdout (no GPU)")
-    ap.add_argument("--sweep-out", default=os.path.join(ROOT, "gpurun_out", "sweep.jsonl"))
+    ap.add_argument("--sweep-out", default=None, help="file the sweep appends its JSON lines to (default: a new temporary file)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -569,7 +569,10 @@ def main():
         args.workload = f"{args.workload}@d={args.d}"
         WORKLOADS[args.workload] = tuple(w)
     if args.sweep:
-        os.makedirs(os.path.dirname(args.sweep_out), exist_ok=True)
+        if args.sweep_out is None:
+            fd, args.sweep_out = tempfile.mkstemp(prefix="draco_sweep_", suffix=".jsonl")
+            os.close(fd)
+        os.makedirs(os.path.dirname(os.path.abspath(args.sweep_out)), exist_ok=True)
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -62,19 +62,5 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
-def build_probe() -> str:
-    """Compile the stand-alone bandwidth probe (csrc/bw_probe.cu) to paper_1803_09877_b200/bw_probe."""
-    out = os.path.join(PKG, "bw_probe")
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-o", out,
-           os.path.join(CSRC, "bw_probe.cu")]
-    r = subprocess.run(cmd, capture_output=True, text=True)
-    if r.returncode != 0:
-        raise RuntimeError("nvcc failed: " + " ".join(cmd) + "\n" + r.stdout + r.stderr)
-    return out
-
-
 if __name__ == "__main__":
-    if "--probe" in sys.argv:
-        print(build_probe())
-    else:
-        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
