@@ -272,11 +272,12 @@ cyc_encode_stream_kernel(const float* __restrict__ G, float2* __restrict__ Z, in
 }
 
 // Any s, any length / alignment: one coordinate per thread, rows re-read through the caches,
-// fp64 accumulation throughout.  half > 0: packed mode (len complex coordinates; the imaginary
+// fp64 taps and fp64 accumulation throughout (a tap rounded to fp32 is a fixed error of 2^-24 |tap| that
+// the decoder's cancellation amplifies like any other).  half > 0: packed mode (len complex coordinates; the imaginary
 // parts come from G[r][half + i], zero beyond d_real).
 __global__ void __launch_bounds__(kGenericThreads)
 cyc_encode_generic_kernel(const float* __restrict__ G, float2* __restrict__ Z, int64_t len, int64_t ldg, int64_t ldz,
-                          int64_t half, int64_t d_real, int n, int s, const float2* __restrict__ taps,
+                          int64_t half, int64_t d_real, int n, int s, const double2* __restrict__ taps,
                           const __grid_constant__ EncodePhase64 ph) {
     const int64_t stride = (int64_t)gridDim.x * kGenericThreads;
     for (int64_t i = (int64_t)blockIdx.x * kGenericThreads + threadIdx.x; i < len; i += stride) {
@@ -286,14 +287,14 @@ cyc_encode_generic_kernel(const float* __restrict__ G, float2* __restrict__ Z, i
             for (int t = 0; t <= 2 * s; ++t) {
                 int r = j - t;
                 if (r < 0) r += n;
-                const float2 c = taps[t];
+                const double2 c = taps[t];
                 const double g = (double)G[(int64_t)r * ldg + i];
-                ar = fma((double)c.x, g, ar);
-                ai = fma((double)c.y, g, ai);
+                ar = fma(c.x, g, ar);
+                ai = fma(c.y, g, ai);
                 if (has_b) {
                     const double gb = (double)G[(int64_t)r * ldg + half + i];
-                    br = fma((double)c.x, gb, br);
-                    bi = fma((double)c.y, gb, bi);
+                    br = fma(c.x, gb, br);
+                    bi = fma(c.y, gb, bi);
                 }
             }
             const double2 rot = ph.phase[j];

@@ -61,7 +61,7 @@ void build_groups(int n, int s, GroupTable* gt) {
 // Cyclic code tables.  W[j][k] = n^(-1/2) prod_{m in alpha_j} (w^k - w^m) with
 // alpha_j = {j+2s+1 .. j+n-1} (mod n): the monic polynomial of degree n-2s-1 that the
 // construction [q_j 1][C_L]_{.,alpha_j} = 0 defines, evaluated at w^k.
-int build_cyclic_tables(draco_plan* p, std::vector<float2>* taps_full, std::vector<double2>* twiddle) {
+int build_cyclic_tables(draco_plan* p, std::vector<double2>* taps_full, std::vector<double2>* twiddle) {
     const int n = p->n, s = p->s, M = n - 2 * s - 1;
     std::vector<cld> w0(2 * s + 1);
     const long double rsn = 1.0L / sqrtl((long double)n);
@@ -87,10 +87,10 @@ int build_cyclic_tables(draco_plan* p, std::vector<float2>* taps_full, std::vect
     memset(&p->phase64, 0, sizeof(p->phase64));
     for (int t = 0; t <= 2 * s; ++t) {
         const cld v = root_of_unity(n, -(long long)t * M) * w0[t];
-        (*taps_full)[t] = make_float2((float)v.real(), (float)v.imag());
+        (*taps_full)[t] = make_double2((double)v.real(), (double)v.imag());
         if (t < kMaxTaps) {
-            p->taps.tap[t] = (*taps_full)[t];
-            p->taps64.tap[t] = make_double2((double)v.real(), (double)v.imag());
+            p->taps.tap[t] = make_float2((float)v.real(), (float)v.imag());
+            p->taps64.tap[t] = (*taps_full)[t];
         }
     }
     memset(&p->phase, 0, sizeof(p->phase));
@@ -148,7 +148,7 @@ int draco_plan_create(int n, int s, int64_t d, int code, draco_plan** out) {
     if (err != cudaSuccess) { free_plan(p); return cuda_fail(err, "cudaGetDevice"); }
 
     int rc = DRACO_OK;
-    std::vector<float2> taps_full;
+    std::vector<double2> taps_full;
     std::vector<double2> twiddle;
     if (code == DRACO_REP) {
         build_groups(n, s, &p->groups);
@@ -172,8 +172,8 @@ int draco_plan_create(int n, int s, int64_t d, int code, draco_plan** out) {
         DRACO_TRY(cudaMalloc(&p->cyc_dev, sizeof(CycDevice)));
         DRACO_TRY(cudaMemset(p->cyc_dev, 0, sizeof(CycDevice)));
         DRACO_TRY(cudaMemcpy(p->cyc_dev, twiddle.data(), sizeof(double2) * kMaxN, cudaMemcpyHostToDevice));
-        DRACO_TRY(cudaMalloc(&p->taps_full_dev, sizeof(float2) * taps_full.size()));
-        DRACO_TRY(cudaMemcpy(p->taps_full_dev, taps_full.data(), sizeof(float2) * taps_full.size(),
+        DRACO_TRY(cudaMalloc(&p->taps_full_dev, sizeof(double2) * taps_full.size()));
+        DRACO_TRY(cudaMemcpy(p->taps_full_dev, taps_full.data(), sizeof(double2) * taps_full.size(),
                              cudaMemcpyHostToDevice));
         p->project_grid = project_grid_size(p->sm_count, n);
         // per block and node: a double2 partial of e_j, then (after all of those) a double partial of q_j

@@ -82,7 +82,7 @@ struct draco_plan {
     draco::EncodePhase phase;
     draco::EncodeTaps64 taps64;
     draco::EncodePhase64 phase64;
-    float2* taps_full_dev;            // generic encoder: taps for any s, device [2s+1]
+    double2* taps_full_dev;           // generic encoder: fp64 taps for any s, device [2s+1]
     // device scratch
     draco::CycDevice* cyc_dev;
     draco::DeviceInfo* info_dev;

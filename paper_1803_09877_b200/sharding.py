@@ -28,18 +28,40 @@ def locate_sharded(plan, R, f, flags, e_buf, group=None, stream=None):
 
     ``plan`` is the rank's plan for its own slice; ``e_buf`` a float64 tensor of 3 n
     values on the same device as R.  Every rank ends with the same flags.
+
+    ``stream`` (a ``torch.cuda.Stream``, or None for torch's current stream) carries all three
+    steps: the collective is enqueued by torch on its *current* stream, so a given stream is
+    made current for the duration of the call; the all-reduce then sees the projection's result
+    and the solve sees the all-reduce's.
     """
+    import contextlib
+
     import torch.distributed as dist
-    plan.cyc_project(R, f, e_buf, stream=stream)
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
-        dist.all_reduce(e_buf, op=dist.ReduceOp.SUM, group=group)
-    plan.cyc_locate_from_projection(e_buf, flags, stream=stream)
+    if stream is None:
+        ctx = contextlib.nullcontext()
+    else:
+        import torch
+        ctx = torch.cuda.stream(stream)
+    with ctx:
+        plan.cyc_project(R, f, e_buf, stream=stream)
+        if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+            dist.all_reduce(e_buf, op=dist.ReduceOp.SUM, group=group)
+        plan.cyc_locate_from_projection(e_buf, flags, stream=stream)
     return flags
 
 
-def merge_flags(flags, group=None):
-    """Repetition code: a node is flagged if any shard saw it disagree (element-wise MAX)."""
+def merge_flags(flags, group=None, stream=None):
+    """Repetition code: a node is flagged if any shard saw it disagree (element-wise MAX).
+    ``stream``: as in ``locate_sharded`` (the stream the decode that wrote ``flags`` ran on)."""
+    import contextlib
+
     import torch.distributed as dist
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
-        dist.all_reduce(flags, op=dist.ReduceOp.MAX, group=group)
+    if stream is None:
+        ctx = contextlib.nullcontext()
+    else:
+        import torch
+        ctx = torch.cuda.stream(stream)
+    with ctx:
+        if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+            dist.all_reduce(flags, op=dist.ReduceOp.MAX, group=group)
     return flags

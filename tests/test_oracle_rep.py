@@ -49,21 +49,17 @@ def test_streaming_majority_against_sort_and_count():
                 assert cand[c] in items[:, c]
 
 
-def test_streaming_majority_literal_loop():
-    """Algorithm 2 run item by item in plain Python on single sequences."""
-    rng = np.random.default_rng(1)
-    for _ in range(200):
-        m = int(rng.integers(1, 12))
-        seq = rng.integers(0, 3, size=m).astype(np.uint32)
-        ma, counter = seq[0], 0
-        for x in seq:
-            if counter == 0:
-                ma, counter = x, 1
-            elif ma == x:
-                counter += 1
-            else:
-                counter -= 1
-        assert orc.majority_stream(seq[:, None])[0] == ma
+def test_streaming_majority_on_every_short_sequence():
+    """Every sequence of up to 7 items over a 3-letter alphabet: whenever one letter holds strictly more than
+    half of the positions the vote returns it, and otherwise it returns a letter that occurs in the sequence."""
+    for m in range(1, 8):
+        seqs = np.array(list(itertools.product(range(3), repeat=m)), dtype=np.uint32).T      # [m][3^m]
+        cand = orc.majority_stream(seqs)
+        counts = np.stack([(seqs == v).sum(axis=0) for v in range(3)])                        # [3][3^m]
+        has_majority = 2 * counts.max(axis=0) > m
+        assert has_majority.any() and (m < 2 or (~has_majority).any())
+        np.testing.assert_array_equal(cand[has_majority], counts.argmax(axis=0)[has_majority])
+        assert all(cand[c] in seqs[:, c] for c in np.flatnonzero(~has_majority))
 
 
 def test_encode_replicas_identical_and_equal_group_sum():

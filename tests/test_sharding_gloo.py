@@ -1,4 +1,4 @@
-"""The d-sharded path on two CPU ranks (gloo): the sharding helpers and the one exchange,
+"""The d-sharded path on two and three CPU ranks (gloo): the sharding helpers and the one exchange,
 with the oracle standing in for the kernels behind the plan interface."""
 import os
 import socket
@@ -63,8 +63,9 @@ def _worker(rank, world, port, n, s, d, adv, result):
     dist.destroy_process_group()
 
 
-def test_two_rank_sharded_locate_and_decode():
-    n, s, d, world = 15, 2, 10_000, 2
+@pytest.mark.parametrize("world,d", [(2, 10_000), (3, 9_001)])       # 3 ranks: shards of 4096, 4096 and 809 coordinates
+def test_sharded_locate_and_decode(world, d):
+    n, s = 15, 2
     adv = [3, 11]
     with socket.socket() as sock:
         sock.bind(("127.0.0.1", 0))
@@ -85,5 +86,42 @@ def test_two_rank_sharded_locate_and_decode():
         np.testing.assert_allclose(e[2 * n:], orc.cyc_project_energy(R), rtol=1e-10)
         exact = G[:, c0:c1].astype(np.float64).sum(axis=0)
         assert np.abs(u - exact).max() <= 1e-4 * np.abs(exact).max()
-        assert rep_flags.tolist()[:2] == [1, 1] and rep_flags.sum() == 2
-    np.testing.assert_array_equal(result[0][1], result[1][1])          # every rank holds the same e
+        assert rep_flags.tolist()[:world] == [1] * world and rep_flags.sum() == world
+    for r in range(1, world):
+        np.testing.assert_array_equal(result[0][1], result[r][1])      # every rank holds the same e
+    sizes = [result[r][3][1] - result[r][3][0] for r in range(world)]
+    assert sum(sizes) == d and (world == 2 or len(set(sizes)) > 1)     # the 3-rank case has uneven shards
+
+
+def test_a_given_stream_is_made_current_around_the_collective(monkeypatch):
+    """locate_sharded(stream=...) runs projection, all-reduce and solve with that stream as torch's current one
+    (the collective is enqueued on the current stream, whatever stream the kernels were given)."""
+    import contextlib
+
+    from paper_1803_09877_b200 import sharding
+    events = []
+
+    @contextlib.contextmanager
+    def fake_stream_ctx(stream):
+        events.append(("enter", stream))
+        yield
+        events.append(("exit", stream))
+
+    class RecordingPlan:
+        def cyc_project(self, R, f, e, stream=None):
+            events.append(("project", stream))
+
+        def cyc_locate_from_projection(self, e, flags, stream=None):
+            events.append(("solve", stream))
+
+    monkeypatch.setattr(torch.cuda, "stream", fake_stream_ctx)
+    token = object()
+    flags = torch.zeros(4, dtype=torch.uint8)
+    sharding.locate_sharded(RecordingPlan(), None, None, flags, None, stream=token)
+    assert events == [("enter", token), ("project", token), ("solve", token), ("exit", token)]
+    events.clear()
+    sharding.merge_flags(flags, stream=token)
+    assert events == [("enter", token), ("exit", token)]
+    events.clear()
+    sharding.locate_sharded(RecordingPlan(), None, None, flags, None)          # no stream: nothing is switched
+    assert events == [("project", None), ("solve", None)]
