@@ -186,7 +186,10 @@ int draco_cyc_locate_from_projection(draco_plan* plan, const double* e, uint8_t*
  * Limits: n <= DRACO_MAX_N (128) and device ordinal < 64, else DRACO_ELIMIT; d is unbounded
  * (at most 296 blocks are launched, each walking its share of the tiles).
  * The first call on each device looks up the array's device address (with that device current);
- * make that first call before any stream capture begins.  All calls on a device share the one
+ * make that first call before any stream capture begins.  The CUDA runtime may place the library's
+ * kernels and this array in device memory only then (lazy module loading), so where another allocator
+ * is about to take the whole device, make one call on it (any small input) before that happens: a
+ * first call on a device with no memory left fails with DRACO_ECUDA.  All calls on a device share the one
  * array, which keeps the previous call's contents (every call overwrites all entries it reads, so
  * nothing needs clearing); two calls that overlap on the GPU, on any streams, race on it.
  * Same kernel and arithmetic as draco_cyc_project; only the number of fp64 block partials may differ
