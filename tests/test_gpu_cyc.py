@@ -127,8 +127,10 @@ def test_locate_and_decode_parity_on_identical_R(n, s, d, n_adv_mode):
     assert torch.equal(u2, u) and torch.equal(f2, flags)
 
 
+# odd d: the one-coordinate-per-thread encoder (fp64 taps) and the scalar projection / recovery paths
 @pytest.mark.parametrize("n,s,d,bar", [(15, 2, 100_000, 1e-4), (15, 1, 30_000, 1e-4), (45, 5, 30_000, None),
-                                        (45, 3, 30_000, None)])
+                                        (45, 3, 30_000, None), (45, 3, 20_001, None), (45, 5, 20_001, None),
+                                        (20, 8, 10_002, None)])
 def test_pipeline_against_exact_sum(n, s, d, bar):
     """encode -> corrupt -> locate -> decode, all on the device, against G 1_P."""
     dr, plan = _plan(n, s, d)
@@ -328,7 +330,8 @@ def test_full_size_decode_on_generated_R_sampled():
 
 # ------------------------------------------------------------------ packed transport (Section 3, last paragraph)
 # (n, s, d): d % 8 == 0 takes the streaming kernel and 64-bit stores; the others the generic paths (odd d pads the last imaginary part)
-PACKED_SHAPES = [(15, 2, 100_000), (45, 5, 24_592), (45, 3, 6152), (15, 2, 1001), (9, 1, 6), (15, 7, 4100), (20, 8, 1032)]
+PACKED_SHAPES = [(15, 2, 100_000), (45, 5, 24_592), (45, 3, 6152), (15, 2, 1001), (9, 1, 6), (15, 7, 4100), (20, 8, 1032),
+                 (45, 3, 20_001), (45, 5, 20_003)]
 
 
 def _packed_plan(n, s, d):
