@@ -108,6 +108,7 @@ def oracle_step(workload, d_sample, seed):
 
 
 def oracle_threads():
+    """Threads the oracle's numerical libraries (numpy's BLAS) may use right now."""
     try:
         from threadpoolctl import threadpool_info
         infos = threadpool_info()
@@ -116,17 +117,33 @@ def oracle_threads():
         return 1
 
 
-def cpu_baseline(workload, target_seconds=15.0):
+def cpu_baseline(workload, target_seconds=8.0):
+    """The oracle as it stands on a bounded sample of the workload, once with every host core its libraries take
+    and once limited to one thread (the two figures the measurement plan names), core count stated."""
     code, n, s, d, std, models, params = WORKLOADS[workload]
     probe = min(d, 200_000)
     oracle_step(workload, probe, SEED)                                   # builds and caches the code tables
     dt, _ = oracle_step(workload, probe, SEED)
     d_sample = int(min(d, max(probe, probe * target_seconds / max(dt, 1e-3))))
-    dt, ok = oracle_step(workload, d_sample, SEED)
+    dt_all, ok = oracle_step(workload, d_sample, SEED)
+    cores = oracle_threads()
+    dt_one = None
+    try:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            dt_one, ok1 = oracle_step(workload, d_sample, SEED)
+        ok = ok and ok1
+    except Exception:
+        pass
     per = 8 if code == "cyc" else 4                      # coded bytes per gradient coordinate (packed: 8 per 2)
-    return {"value": per * n * d_sample / dt / 1e9, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-            "sample": f"first {d_sample} of {d} coordinates, all {n} workers, one pass in {dt:.2f} s "
-                      f"(numpy fp64/complex128; flags correct: {ok})"}
+    out = {"value": per * n * d_sample / dt_all / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "host_cores": os.cpu_count(),
+           "sample": f"first {d_sample} of {d} coordinates, all {n} workers, one pass in {dt_all:.2f} s with {cores} threads"
+                     + (f" and {dt_one:.2f} s with 1 thread" if dt_one else "")
+                     + f" (numpy fp64/complex128; flags correct: {ok})"}
+    if dt_one:
+        out["value_1_thread"] = per * n * d_sample / dt_one / 1e9
+    return out
 
 
 def run_reference(args):
@@ -216,20 +233,27 @@ class ClockSampler:
         return out
 
 
-def run_gpu(args):
+def stage_launches(code, n, n_adv):
+    """Kernels launched per step: encode 1; corrupt 1 (all adversaries in one launch); cyclic locate = projection
+    (two launches over half the rows each when n > 64) + reduction of the block partials fused with the solve;
+    decode = decode vector + recovery (repetition: vote + finish, no separate locate)."""
+    cyc = code in ("cyc", "cycp")
+    return {"encode": 1, "corrupt": 1 if n_adv else 0, "locate": ((2 if n > 64 else 1) + LOCATE_TAIL_LAUNCHES) if cyc else 0,
+            "decode": 2}
+
+
+LOCATE_TAIL_LAUNCHES = 2     # cyc_reduce_partials_kernel, cyc_solve_kernel
+
+
+def measure_workload(args, workload, world, rank, with_graph, with_e2e):
+    """Times `args.steps` steps of one workload on this rank's GPU (inputs resident in HBM) and, optionally, the
+    CUDA-graph replay and the host-buffer pipeline.  Returns the pieces of the JSON line."""
     import torch
     import torch.distributed as dist
 
     import paper_1803_09877_b200 as dr
     from paper_1803_09877_b200.sharding import locate_sharded, merge_flags
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    workload = args.workload
     code, n, s, d, std, models, params = WORKLOADS[workload]
     cyc = code in ("cyc", "cycp")
     packed = code == "cycp"
@@ -237,6 +261,7 @@ def run_gpu(args):
     adv, model, param = adversaries(workload)
     plan = dr.Plan(n, s, d, dr.CYC_PACKED if packed else dr.CYC if cyc else dr.REP)
     stream = torch.cuda.current_stream()
+    steps, warmup = args.steps, max(args.warmup, 3)
 
     # inputs resident in HBM; rank r holds coordinates [r d, (r+1) d) of a d * world vector
     G = torch.empty((n, d), dtype=torch.float32, device="cuda")
@@ -280,21 +305,21 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(warmup):
         step()
     sync_all()
     got = sorted(np.flatnonzero(flags.cpu().numpy()).tolist())
     if got != adv.tolist():
-        raise SystemExit(f"flags {got} differ from the planted adversaries {adv.tolist()}")
+        raise SystemExit(f"{workload}: flags {got} differ from the planted adversaries {adv.tolist()}")
 
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
     sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
     time.sleep(0.3)
     sync_all()
     t_start = torch.cuda.Event(enable_timing=True)
     t_stop = torch.cuda.Event(enable_timing=True)
     t_start.record(stream)
-    for k in range(args.steps):
+    for k in range(steps):
         step(events[k])
     t_stop.record(stream)
     sync_all()
@@ -304,8 +329,8 @@ def run_gpu(args):
         t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
-    per_step = {nm: [events[k][i].elapsed_time(events[k][i + 1]) for k in range(args.steps)] for i, nm in enumerate(names)}
+    ms_per_step = total_ms / steps
+    per_step = {nm: [events[k][i].elapsed_time(events[k][i + 1]) for k in range(steps)] for i, nm in enumerate(names)}
     stage_ms = {nm: statistics.mean(v) for nm, v in per_step.items()}
     stage_min = {nm: min(v) for nm, v in per_step.items()}
     stage_med = {nm: statistics.median(v) for nm, v in per_step.items()}
@@ -320,8 +345,9 @@ def run_gpu(args):
     achieved = ab[dom] / (stage_ms[dom] * 1e-3) / 1e9
     # DRAM bytes per gradient coordinate of the dominant kernel, from the ncu captures summarised under profiles/
     # (dram__bytes_read.sum + dram__bytes_write.sum at d = 4 M / 8 M; every byte is touched once, so traffic scales with d).
-    # Valid for n = 45 with the configured s only; null for any other shape.
-    traffic_per_coord = {("cyc", 45, 5): 525.1, ("cycp", 45, 5): 353.6, ("rep", 45, 3): 183.0}.get((code, n, s))
+    # Valid for n = 45 with the configured s only; null for any other shape, and null for a kernel that has changed
+    # since its counters were taken.
+    traffic_per_coord = DOMINANT_TRAFFIC_PER_COORD.get((code, n, s))
     traffic = traffic_per_coord * d if traffic_per_coord else None
     stages = {}
     for nm in names:
@@ -332,13 +358,19 @@ def run_gpu(args):
                           "frac_of_nominal_8TBps": round(g / 8000.0, 4)}
         else:
             stages[nm] = {"ms": round(stage_ms[nm], 4)}
-    # encode 1, corrupt 1 per adversary, cyclic locate = projection (two launches over half the rows each when n > 64)
-    # + reduction of the block partials + solve, decode = decode vector + recovery (repetition: vote + finish)
-    launches = (1 + len(adv) + ((3 + (1 if n > 64 else 0)) if cyc else 0) + 2) * args.steps
+    launches = sum(stage_launches(code, n, len(adv)).values()) * steps
+    roofline = {"bound": "hbm", "kernel": dom_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
+                "algorithmic_bytes_per_launch": ab[dom], "avg_launch_ms": stage_ms[dom]}
+    config = {"workload": workload, "code": code, "n": n, "s": s, "d_per_gpu": d, "adversaries": len(adv),
+              "adversary_models": models, "l2": "inputs larger than L2 (no flush needed)"
+              if ab["coded"] > 4e8 else "working set near L2 size: not an HBM number",
+              "value_is": "bytes of coded gradients (n d complex64 / fp32) per step / step time"}
 
     # the same step captured once into a CUDA graph and replayed (one GPU only: the sharded step has a collective)
     graph_replay = None
-    if world == 1 and not args.no_graph:
+    if with_graph and world == 1:
         side = torch.cuda.Stream()
         side.wait_stream(stream)
         cg = torch.cuda.CUDAGraph()
@@ -351,21 +383,21 @@ def run_gpu(args):
         sync_all()
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record(stream)
-        for _ in range(args.steps):
+        for _ in range(steps):
             cg.replay()
         g1.record(stream)
         sync_all()
         got = sorted(np.flatnonzero(flags.cpu().numpy()).tolist())
         if got != adv.tolist():
             raise SystemExit(f"graph replay: flags {got} differ from the planted adversaries {adv.tolist()}")
-        gms = g0.elapsed_time(g1) / args.steps
+        gms = g0.elapsed_time(g1) / steps
         graph_replay = {"ms_per_step": gms, "value": ab["coded"] / (gms * 1e-3) / 1e9, "unit": UNIT,
                         "stream_launch_ms_per_step": ms_per_step}
         del cg
 
     # end to end through the host-buffer entry point (rank-local; H2D of G and f, D2H of u and flags)
     e2e = None
-    if not args.no_e2e:
+    if with_e2e:
         del events
         Gh = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
         Gh.copy_(G)
@@ -375,12 +407,12 @@ def run_gpu(args):
         uh = torch.empty(d, dtype=torch.float32, pin_memory=True)
         flh = torch.empty(n, dtype=torch.uint8, pin_memory=True)
         torch.cuda.synchronize()
-        reps = max(2, min(args.steps, 5))
+        reps = max(2, min(steps, 5))
         plan.pipeline_host(Gh, fh if cyc else None, adv, model, param, SEED + 2, Z, uh, flh)   # warm-up, allocs
         sync_all()
         t0 = time.perf_counter()
         for _ in range(reps):
-            info = plan.pipeline_host(Gh, fh if cyc else None, adv, model, param, SEED + 2, Z, uh, flh)
+            plan.pipeline_host(Gh, fh if cyc else None, adv, model, param, SEED + 2, Z, uh, flh)
         sync_all()
         dt = (time.perf_counter() - t0) / reps
         if world > 1:
@@ -392,23 +424,65 @@ def run_gpu(args):
         e2e = {"value": ab["coded"] * world / dt / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": 4 * n * d + (4 * vlen if cyc else 0), "d2h_bytes_per_step": 4 * d + n,
                "ms_per_step": dt * 1e3, "steps": reps}
+        del Gh, fh, uh, flh
+    out = {"value": value, "ms_per_step": ms_per_step, "config": config, "roofline": roofline, "stages": stages,
+           "clocks": clocks, "e2e": e2e, "graph_replay": graph_replay, "gpu_launches": launches,
+           "dtype": "f32 (complex64 vectors; f64 centre taps, projection sums and recovery)" if cyc
+           else "f32 (u32 bit patterns in the vote)"}
+    plan.close()
+    del G, Z, u, f, flags, e
+    torch.cuda.empty_cache()
+    return out
 
+
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per gradient coordinate of the dominant kernel (profiles/)
+DOMINANT_TRAFFIC_PER_COORD = {("cyc", 45, 5): 525.1, ("cycp", 45, 5): 353.6, ("rep", 45, 3): 183.0}
+SECONDARY_WORKLOADS = ["rep_n45_s3_d11.7M", "cycp_n45_s5_d60.2M"]
+
+
+def launch_plan(args, argv):
+    """How `bench.py --gpus N` starts its N ranks when it was not itself started by torchrun: the command and the
+    extra environment of one torchrun process group on this node (rendezvous on 127.0.0.1)."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--standalone", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--local-addr", "127.0.0.1", os.path.abspath(__file__)] + [a for a in argv if a != "--dry-run"]
+    env = {"MASTER_ADDR": "127.0.0.1", "OMP_NUM_THREADS": "1"}
+    return cmd, env
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    ranks = None
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        mine = {"rank": rank, "device": local, "uuid": str(torch.cuda.get_device_properties(local).uuid)}
+        gathered = [None] * world
+        dist.all_gather_object(gathered, mine)
+        ranks = gathered
+        if len({g["uuid"] for g in gathered}) != world:
+            raise SystemExit(f"ranks share a GPU: {gathered}")
+    main = measure_workload(args, args.workload, world, rank, with_graph=not args.no_graph, with_e2e=not args.no_e2e)
+    secondary = None
+    if world == 1 and not args.no_secondary and args.workload == DEFAULT_WORKLOAD:
+        secondary = {}
+        for wl in SECONDARY_WORKLOADS:
+            r = measure_workload(args, wl, world, rank, with_graph=False, with_e2e=False)
+            secondary[wl] = {"value": r["value"], "unit": UNIT, "ms_per_step": r["ms_per_step"], "stages": r["stages"],
+                             "roofline": r["roofline"], "gpu_launches": r["gpu_launches"], "clocks": r["clocks"],
+                             "config": r["config"]}
     if rank == 0:
-        cb = cpu_baseline(workload) if (world == 1 and not args.no_cpu_baseline) else None
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32 (complex64 vectors; f64 centre taps, projection sums and recovery)"
-                if cyc else "f32 (u32 bit patterns in the vote)", "data": "synthetic",
-                "config": {"workload": workload, "code": code, "n": n, "s": s, "d_per_gpu": d, "adversaries": len(adv),
-                           "adversary_models": models, "l2": "inputs larger than L2 (no flush needed)"
-                           if ab["coded"] > 4e8 else "working set near L2 size: not an HBM number",
-                           "value_is": "bytes of coded gradients (n d complex64 / fp32) per step / step time"},
-                "roofline": {"bound": "hbm", "kernel": dom_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
-                             "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
-                             "algorithmic_bytes_per_launch": ab[dom], "avg_launch_ms": stage_ms[dom]},
-                "stages": stages, "clocks": clocks, "e2e": e2e, "graph_replay": graph_replay, "gpu_launches": launches,
-                "cpu_baseline": cb}
+        cb = cpu_baseline(args.workload) if (world == 1 and not args.no_cpu_baseline) else None
+        line = {"metric": METRIC, "value": main["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": main["ms_per_step"], "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": main["dtype"], "data": "synthetic",
+                "config": main["config"], "roofline": main["roofline"], "stages": main["stages"], "clocks": main["clocks"],
+                "e2e": main["e2e"], "graph_replay": main["graph_replay"], "gpu_launches": main["gpu_launches"],
+                "cpu_baseline": cb, "secondary": secondary, "ranks": ranks}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -491,16 +565,17 @@ def run_sweep(args):
                         checks[label] = {"planted": len(adv), "flags_match": got == sorted(adv), "err": err,
                                          "status": info["status"], "no_majority": info["no_majority"]}
                     adv = di.choose_adversaries(seed + 1, n, s).tolist()
-                    enc_ms = timed(lambda: plan.encode(G, Z))
+                    reps = 20 if d >= 11_000_000 else 5
+                    enc_ms = timed(lambda: plan.encode(G, Z), reps)
                     if adv:
                         plan.corrupt(Z, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 4)
-                    dec_ms = timed(lambda: plan.locate_decode(Z, f if cyc else None, flags, u))
+                    dec_ms = timed(lambda: plan.locate_decode(Z, f if cyc else None, flags, u), reps)
                     ab = algorithmic_bytes(code, n, s, d, len(adv))
                     enc_hbm = ab["encode"] / (enc_ms * 1e-3) / 1e9
                     dec_hbm = (ab["locate"] + ab["decode"]) / (dec_ms * 1e-3) / 1e9
                     tol = 1e-5 if not cyc else (1e-4 if n <= 15 else None)
                     ok_s = checks["s"]["flags_match"] and checks["0"]["flags_match"]
-                    line = {"code": code, "n": n, "s": s, "d": d, "encode_ms": enc_ms, "decode_ms": dec_ms,
+                    line = {"code": code, "n": n, "s": s, "d": d, "encode_ms": enc_ms, "decode_ms": dec_ms, "timed_reps": reps,
                             "coded_GBps_produced": ab["coded"] / (enc_ms * 1e-3) / 1e9,
                             "coded_GBps_consumed": ab["coded"] / (dec_ms * 1e-3) / 1e9,
                             "encode_hbm_GBps": enc_hbm, "encode_frac": enc_hbm / peak,
@@ -559,6 +634,9 @@ def main():
     ap.add_argument("--sweep-out", default=None, help="file the sweep appends its JSON lines to (default: a new temporary file)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the repetition-code and packed-transport workloads "
+                    "that follow the default workload on one GPU")
+    ap.add_argument("--dry-run", action="store_true", help="print how N ranks would be launched (JSON) and exit")
     args = ap.parse_args()
     if args.sweep_table:
         sys.stdout.write(sweep_table(args.sweep_table))
@@ -568,6 +646,17 @@ def main():
         w[3] = args.d
         args.workload = f"{args.workload}@d={args.d}"
         WORKLOADS[args.workload] = tuple(w)
+    if (args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.sweep and args.impl == "ours") or args.dry_run:
+        # started by hand as `python bench.py --gpus N`: become N ranks, one per GPU, under torchrun
+        cmd, env = launch_plan(args, sys.argv[1:])
+        if args.dry_run:
+            single = [sys.executable, os.path.abspath(__file__)] + [a for a in sys.argv[1:] if a != "--dry-run"]
+            print(json.dumps({"launch": cmd if (args.gpus > 1 and args.impl == "ours") else single,
+                              "env": env if (args.gpus > 1 and args.impl == "ours") else {},
+                              "ranks": args.gpus if args.impl == "ours" else 1}))
+            return
+        os.environ.update(env)
+        os.execvp(cmd[0], cmd)
     if args.sweep:
         if args.sweep_out is None:
             fd, args.sweep_out = tempfile.mkstemp(prefix="draco_sweep_", suffix=".jsonl")

@@ -226,7 +226,8 @@ int draco_pipeline_host(draco_plan* plan, const float* G_host, const float* f_ho
 int draco_generate(float* out, int rows, int64_t len, int row0, float mean, float std, uint64_t seed, void* stream);
 
 /*
- * The adversary: R = Z + N in place, N non-zero on rows adv_idx[0 .. n_adv-1] (host arrays).
+ * The adversary: R = Z + N in place, N non-zero on rows adv_idx[0 .. n_adv-1] (host arrays, distinct
+ * node indices; all rows are rewritten by one kernel launch).
  *   DRACO_ADV_REVGRAD: row <- -c * row          (param = c)
  *   DRACO_ADV_CONST:   row <- kappa             (param = kappa; imaginary parts 0)
  *   DRACO_ADV_GAUSS:   row <- row + sigma * x   (param = sigma; x from the generator above with

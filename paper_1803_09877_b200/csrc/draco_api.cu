@@ -326,15 +326,15 @@ static int corrupt_range(const draco_plan* plan, void* R, int64_t c0, int64_t le
                          const int* adv_model, const float* adv_param, int n_adv, uint64_t seed, cudaStream_t st) {
     const bool cplx = is_cyc(plan);
     const int64_t per = cplx ? 2 : 1;
+    if (n_adv > plan->n) return DRACO_EINVAL;
+    bool seen[kMaxN] = {};
     for (int a = 0; a < n_adv; ++a) {
-        const int j = adv_idx[a];
-        if (j < 0 || j >= plan->n) return DRACO_EINVAL;
+        if (adv_idx[a] < 0 || adv_idx[a] >= plan->n || seen[adv_idx[a]]) return DRACO_EINVAL;   // all rows go in one launch
+        seen[adv_idx[a]] = true;
         if (adv_model[a] < DRACO_ADV_REVGRAD || adv_model[a] > DRACO_ADV_GAUSS) return DRACO_EINVAL;
-        float* row = (float*)R + ((int64_t)j * ld + c0) * per;
-        int rc = launch_corrupt_row(row, len * per, c0 * per, adv_model[a], adv_param[a], seed, j, cplx, st);
-        if (rc != DRACO_OK) return rc;
     }
-    return DRACO_OK;
+    return launch_corrupt((float*)R, ld * per, len * per, c0 * per, adv_idx, adv_model, adv_param, n_adv, seed, cplx,
+                          plan->sm_count, st);
 }
 
 int draco_corrupt(const draco_plan* plan, void* R, const int* adv_idx, const int* adv_model, const float* adv_param,

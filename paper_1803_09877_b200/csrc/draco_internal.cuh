@@ -126,8 +126,8 @@ int launch_cyc_recover(draco_plan* p, const float2* R, int64_t len, int64_t ld, 
                        cudaStream_t st, float* w = nullptr, float scale = 0.0f);
 int launch_generate(float* out, int rows, int64_t len, int64_t ld, int64_t i0, int row0, float mean, float std,
                     uint64_t seed, cudaStream_t st);
-int launch_corrupt_row(float* row, int64_t nvals, int64_t v0, int model, float param, uint64_t seed, int node,
-                       bool is_complex, cudaStream_t st);
+int launch_corrupt(float* R, int64_t row_pitch, int64_t nvals, int64_t v0, const int* node, const int* model,
+                   const float* param, int n_adv, uint64_t seed, bool is_complex, int sm_count, cudaStream_t st);
 int project_grid_size(int sm_count);
 int project_grid_size(int sm_count, int n);
 

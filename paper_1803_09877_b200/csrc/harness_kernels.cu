@@ -51,11 +51,24 @@ __device__ __forceinline__ float corrupt_value(float v, int64_t idx, int model, 
     return __fadd_rn(v, __fmul_rn(approx_normal(key, (uint64_t)idx, inv_sigma), param));
 }
 
-// One adversarial row, in place; VEC = 4 when the row slice is 16-byte aligned and a multiple of 4 values.
+// All adversarial rows in one launch, in place: blockIdx.y picks the adversary, blockIdx.x strides over its row
+// slice.  VEC = 4 when every row slice is 16-byte aligned and a multiple of 4 values long.
+struct CorruptTable {
+    int32_t node[kMaxN];
+    int32_t model[kMaxN];
+    float param[kMaxN];
+    unsigned long long key[kMaxN];        // generator key of the node's noise row
+};
+
 template <int VEC>
 __global__ void __launch_bounds__(kThreads)
-corrupt_kernel(float* __restrict__ row, int64_t nvals, int64_t v0, int model, float param, uint64_t key, int is_complex,
-               float inv_sigma) {
+corrupt_kernel(float* __restrict__ R, int64_t row_pitch, int64_t nvals, int64_t v0, int is_complex, float inv_sigma,
+               const __grid_constant__ CorruptTable tab) {
+    const int a = blockIdx.y;
+    const int model = tab.model[a];
+    const float param = tab.param[a];
+    const uint64_t key = tab.key[a];
+    float* row = R + (int64_t)tab.node[a] * row_pitch + v0;
     const int64_t stride = (int64_t)gridDim.x * kThreads;
     if (VEC == 4) {
         float4* row4 = reinterpret_cast<float4*>(row);
@@ -83,32 +96,49 @@ uint64_t host_splitmix64_at(uint64_t seed, uint64_t ctr) {
     return z ^ (z >> 31);
 }
 
-int grid_for(int64_t work) {
+int grid_for(int64_t work, int sm_count, int per_sm) {
     int64_t want = (work + kThreads - 1) / kThreads;
-    if (want > 148 * 16) want = 148 * 16;
+    const int64_t cap = (int64_t)(sm_count > 0 ? sm_count : 1) * per_sm;
+    if (want > cap) want = cap;
     if (want < 1) want = 1;
     return (int)want;
+}
+
+int device_sm_count() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 1;
+    return sms;
 }
 
 }  // namespace
 
 int launch_generate(float* out, int rows, int64_t len, int64_t ld, int64_t i0, int row0, float mean, float sd,
                     uint64_t seed, cudaStream_t st) {
-    generate_kernel<<<grid_for(len), kThreads, 0, st>>>(out, rows, len, ld, i0, row0, mean, sd, seed, inv_sigma_f32());
+    generate_kernel<<<grid_for(len, device_sm_count(), 16), kThreads, 0, st>>>(out, rows, len, ld, i0, row0, mean, sd, seed,
+                                                                              inv_sigma_f32());
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }
 
-int launch_corrupt_row(float* row, int64_t nvals, int64_t v0, int model, float param, uint64_t seed, int node,
-                       bool is_complex, cudaStream_t st) {
-    const uint64_t key = host_splitmix64_at(seed, (uint64_t)node);
-    const bool vec4 = (nvals % 4 == 0) && ((reinterpret_cast<uintptr_t>(row) & 15u) == 0);
-    if (vec4)
-        corrupt_kernel<4><<<grid_for(nvals / 4), kThreads, 0, st>>>(row, nvals, v0, model, param, key, is_complex ? 1 : 0,
-                                                                    inv_sigma_f32());
-    else
-        corrupt_kernel<1><<<grid_for(nvals), kThreads, 0, st>>>(row, nvals, v0, model, param, key, is_complex ? 1 : 0,
-                                                                inv_sigma_f32());
+// R = Z + N on the rows node[0 .. n_adv-1]: values [v0, v0 + nvals) of each (fp32 values; a complex entry is two).
+int launch_corrupt(float* R, int64_t row_pitch, int64_t nvals, int64_t v0, const int* node, const int* model,
+                   const float* param, int n_adv, uint64_t seed, bool is_complex, int sm_count, cudaStream_t st) {
+    if (n_adv == 0) return DRACO_OK;
+    CorruptTable tab;
+    for (int a = 0; a < n_adv; ++a) {
+        tab.node[a] = node[a];
+        tab.model[a] = model[a];
+        tab.param[a] = param[a];
+        tab.key[a] = host_splitmix64_at(seed, (uint64_t)node[a]);
+    }
+    const bool vec4 = (nvals % 4 == 0) && (row_pitch % 4 == 0) && (v0 % 4 == 0) && ((reinterpret_cast<uintptr_t>(R) & 15u) == 0);
+    // enough blocks per adversary that all of them together fill the device about sixteen times over
+    int per_sm = 16 / n_adv;
+    if (per_sm < 2) per_sm = 2;
+    const dim3 grid(grid_for(vec4 ? nvals / 4 : nvals, sm_count, per_sm), n_adv);
+    if (vec4) corrupt_kernel<4><<<grid, kThreads, 0, st>>>(R, row_pitch, nvals, v0, is_complex ? 1 : 0, inv_sigma_f32(), tab);
+    else corrupt_kernel<1><<<grid, kThreads, 0, st>>>(R, row_pitch, nvals, v0, is_complex ? 1 : 0, inv_sigma_f32(), tab);
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }

@@ -42,3 +42,24 @@ def test_sweep_table_renders_one_row_per_point(tmp_path):
     rows = [ln for ln in out.stdout.splitlines() if ln.startswith("| cyc")]
     assert len(rows) == 2 and "| 15 | 2 | 1.0 M | 0.050 | 3600 (0.55) | 0.080 | 3000 (0.46) | 2400 / 1500 |" in rows[0]
     assert rows[0].rstrip().endswith("| yes | yes |") and "| NO | yes |" in rows[1]
+
+
+def test_gpus_n_started_by_hand_launches_n_ranks_under_torchrun():
+    """`python bench.py --gpus 4` without torchrun's environment re-executes itself as 4 ranks (dry run: the plan only)."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--steps", "3", "--warmup", "3", "--dry-run"],
+                         capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
+    assert out.returncode == 0, out.stderr
+    plan = json.loads(out.stdout.strip())
+    cmd = plan["launch"]
+    assert plan["ranks"] == 4 and cmd[1:3] == ["-m", "torch.distributed.run"]
+    assert "--nproc-per-node=4" in cmd and "--standalone" in cmd and "--dry-run" not in cmd
+    assert cmd[cmd.index("--local-addr") + 1] == "127.0.0.1" and plan["env"]["MASTER_ADDR"] == "127.0.0.1"
+    tail = cmd[cmd.index(os.path.join(ROOT, "bench.py")) + 1:]
+    assert tail == ["--gpus", "4", "--steps", "3", "--warmup", "3"]
+    # one GPU, and the reference arm at any N, start no process group
+    for extra in (["--gpus", "1"], ["--gpus", "4", "--impl", "reference"]):
+        out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--dry-run"] + extra, capture_output=True, text=True,
+                             timeout=120, cwd=ROOT, env=env)
+        plan = json.loads(out.stdout.strip())
+        assert plan["ranks"] == 1 and "torch.distributed.run" not in plan["launch"] and plan["env"] == {}
