@@ -37,6 +37,13 @@ __device__ __forceinline__ double2 cdiv(double2 a, double2 b) {
 __device__ __forceinline__ double cabs2(double2 a) { return a.x * a.x + a.y * a.y; }
 
 // ------------------------------------------------------------------ projection
+// Arithmetic.  f_i and R[j][i] are fp32, so their product has at most 48 significant bits and is exact in fp64:
+// every term enters an fp64 running sum through one fused multiply-add on the converted operands, and the only
+// rounding left is that of fp64 addition (2^-53 per term).  The device's e_j therefore carries the rounding of the
+// complex64 vectors themselves and nothing of its own; products or short runs in fp32 would add about as much
+// again per term (a 16-term fp32 run: three times as much), which the s x s syndrome system amplifies by about
+// sqrt(s): at s = 20 that noise alone reached the rank cutoff and flagged an honest node.
+//
 // q_j = sum_i |R[j][i]|^2 travels with e_j: it is the yardstick of the locator's rank cutoff (rounding R to
 // complex64 perturbs e_j by about 2^-25 (E f^2 q_j)^(1/2), whatever e_j itself cancels to).  A few digits of it
 // are enough: fp32 terms and tile sums, fp64 across tiles.  Layout of the block partials: [grid][n] double2 (e),
@@ -61,16 +68,16 @@ __device__ __forceinline__ double* q_partials(double2* partial, int n) {
     return reinterpret_cast<double*>(partial + (int64_t)gridDim.x * n);
 }
 // Block = 8 warps over one tile of coordinates; warp w owns rows row0 + w, row0 + w + 8, ... of the
-// launch's nrows <= 8 RPW rows; f for the tile sits in shared memory.  Products and short runs (16 terms)
-// in fp32, running sums in fp64.  More than 64 rows take two launches of half the rows each (rows are
+// launch's nrows <= 8 RPW rows; f for the tile sits in shared memory as fp64 (converted once per tile, used by
+// every row).  More than 64 rows take two launches of half the rows each (rows are
 // independent; f is read twice, 1 % more traffic): 16 rows per warp in registers halve the blocks per SM
 // (0.79 of the copy bandwidth at n = 105), and per-lane sums in shared memory left the compiler too few
 // registers to keep its loads in flight once the squared norms were added (0.98 -> 0.68).
 template <int RPW, bool VEC2>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
                    int row0, int nrows, double2* __restrict__ partial, int accumulate) {
-    __shared__ __align__(16) float fs[kProjectTile];
+    __shared__ __align__(16) double fs[kProjectTile];
     __shared__ double qs[kProjectWarps * RPW];           // q of row warp + r * 8, kept by lane 0 of its warp
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     double accr[RPW], acci[RPW];
@@ -85,7 +92,7 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const int64_t c0 = tile * kProjectTile;
         const int cnt = (int)((len - c0) < kProjectTile ? (len - c0) : kProjectTile);
-        for (int i = threadIdx.x; i < kProjectTile; i += kThreads) fs[i] = (i < cnt) ? __ldcs(f + c0 + i) : 0.0f;
+        for (int i = threadIdx.x; i < kProjectTile; i += kThreads) fs[i] = (i < cnt) ? (double)__ldcs(f + c0 + i) : 0.0;
         __syncthreads();
 #pragma unroll
         for (int r = 0; r < RPW; ++r) {
@@ -93,6 +100,7 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
             if (j < row0 + nrows) {
                 const float2* row = R + (int64_t)j * ld + c0;
                 float eq = 0.f;
+                double ar = 0.0, ai = 0.0;
                 if (VEC2 && cnt == kProjectTile) {
                     const float4* row4 = reinterpret_cast<const float4*>(row);
 #pragma unroll 1
@@ -100,27 +108,27 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
                         float4 v[8];
 #pragma unroll
                         for (int q = 0; q < 8; ++q) v[q] = __ldcs(row4 + (step0 + q) * 32 + lane);
-                        float pr = 0.f, pi = 0.f, pq = 0.f;
+                        float pq = 0.f;
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
-                            const float2 ff = *reinterpret_cast<const float2*>(&fs[((step0 + q) * 32 + lane) * 2]);
-                            pr = fmaf(ff.x, v[q].x, pr); pi = fmaf(ff.x, v[q].y, pi);
-                            pr = fmaf(ff.y, v[q].z, pr); pi = fmaf(ff.y, v[q].w, pi);
+                            const double2 ff = *reinterpret_cast<const double2*>(&fs[((step0 + q) * 32 + lane) * 2]);
+                            ar = fma(ff.x, (double)v[q].x, ar); ai = fma(ff.x, (double)v[q].y, ai);
+                            ar = fma(ff.y, (double)v[q].z, ar); ai = fma(ff.y, (double)v[q].w, ai);
                             pq = energy2(v[q], pq);
                         }
-                        accr[r] += (double)pr;
-                        acci[r] += (double)pi;
                         eq += pq;
                     }
                 } else {
                     for (int i = lane; i < cnt; i += 32) {
                         const float2 v = __ldcs(row + i);
-                        const float ff = fs[i];
-                        accr[r] += (double)(ff * v.x);
-                        acci[r] += (double)(ff * v.y);
+                        const double ff = fs[i];
+                        ar = fma(ff, (double)v.x, ar);
+                        ai = fma(ff, (double)v.y, ai);
                         eq = fmaf(v.y, v.y, fmaf(v.x, v.x, eq));
                     }
                 }
+                accr[r] += ar;
+                acci[r] += ai;
                 eq = warp_sum(eq);
                 if (lane == 0) qs[r * kProjectWarps + warp] += (double)eq;
             }
@@ -150,8 +158,8 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
 
 // The same projection for few rows (n <= 16): with one or two rows per warp the block-wide tile
 // barriers of the kernel above dominate, so here every warp works alone on 256-coordinate chunks
-// of all n rows, with f for its chunk in registers (8 values per lane) and no shared memory or
-// barrier in the loop.  Per-lane running sums in fp64 registers (2 n doubles).
+// of all n rows, with f for its chunk in registers (8 values per lane) and no
+// shared memory or barrier in the loop.  Per-lane running sums in fp64 registers (2 n doubles).
 template <bool VEC2>
 __global__ void __launch_bounds__(kThreads, 2)
 cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
@@ -186,39 +194,29 @@ cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict
 #pragma unroll
                         for (int q = 0; q < 4; ++q) vb[q] = __ldcs(rb + q * 32 + lane);
                     }
-                    float pr = 0.f, pi = 0.f, pq = accq[jj];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        pr = fmaf(ff[q].x, va[q].x, pr); pi = fmaf(ff[q].x, va[q].y, pi);
-                        pr = fmaf(ff[q].y, va[q].z, pr); pi = fmaf(ff[q].y, va[q].w, pi);
-                        pq = energy2(va[q], pq);
-                    }
-                    accr[jj] += (double)pr;
-                    acci[jj] += (double)pi;
-                    accq[jj] = pq;
-                    if (two) {
-                        pr = 0.f; pi = 0.f; pq = accq[jj + 1];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            pr = fmaf(ff[q].x, vb[q].x, pr); pi = fmaf(ff[q].x, vb[q].y, pi);
-                            pr = fmaf(ff[q].y, vb[q].z, pr); pi = fmaf(ff[q].y, vb[q].w, pi);
-                            pq = energy2(vb[q], pq);
+                        const double fx = (double)ff[q].x, fy = (double)ff[q].y;     // shared by the two rows
+                        accr[jj] = fma(fx, (double)va[q].x, accr[jj]); acci[jj] = fma(fx, (double)va[q].y, acci[jj]);
+                        accr[jj] = fma(fy, (double)va[q].z, accr[jj]); acci[jj] = fma(fy, (double)va[q].w, acci[jj]);
+                        accq[jj] = energy2(va[q], accq[jj]);
+                        if (two) {
+                            accr[jj + 1] = fma(fx, (double)vb[q].x, accr[jj + 1]); acci[jj + 1] = fma(fx, (double)vb[q].y, acci[jj + 1]);
+                            accr[jj + 1] = fma(fy, (double)vb[q].z, accr[jj + 1]); acci[jj + 1] = fma(fy, (double)vb[q].w, acci[jj + 1]);
+                            accq[jj + 1] = energy2(vb[q], accq[jj + 1]);
                         }
-                        accr[jj + 1] += (double)pr;
-                        acci[jj + 1] += (double)pi;
-                        accq[jj + 1] = pq;
                     }
                 }
             }
         } else {
             for (int i = lane; i < cnt; i += 32) {
-                const float fi = __ldcs(f + c0 + i);
+                const double fi = (double)__ldcs(f + c0 + i);
 #pragma unroll
                 for (int j = 0; j < NMAX; ++j)
                     if (j < n) {
                         const float2 v = __ldcs(R + (int64_t)j * ld + c0 + i);
-                        accr[j] += (double)(fi * v.x);
-                        acci[j] += (double)(fi * v.y);
+                        accr[j] = fma(fi, (double)v.x, accr[j]);
+                        acci[j] = fma(fi, (double)v.y, acci[j]);
                         accq[j] = fmaf(v.y, v.y, fmaf(v.x, v.x, accq[j]));
                     }
             }
