@@ -59,14 +59,20 @@ enum {
     DRACO_EINTERNAL = -5, /* a bounded wait inside a kernel expired (reported by draco_get_info); results are invalid.
                              Kept for ABI stability: the current kernels contain no such wait and never report it */
     DRACO_ELIMIT = -6,   /* a size exceeds a fixed capacity of the entry point called (see draco_cyc_project_noalloc) */
-    DRACO_ENOMAJ = 1     /* warning: some (group, coordinate) had no strict majority; u holds Algorithm 2's candidate */
+    DRACO_ENOMAJ = 1,    /* warning: some (group, coordinate) had no strict majority; u holds Algorithm 2's candidate */
+    DRACO_EUNSURE = 2    /* warning (cyclic): a self-check of the decoder failed, so V or u may be wrong: the flagged and
+                            the unflagged |t_j| are less than a factor 10 apart (locator_margin), or the recovered u-hat has
+                            an imaginary part above 1e-2 of its real part (im_residual, re_max), or the singular-value
+                            iteration of the syndrome system stopped at its sweep limit (svd_sweeps < 0).  More than s
+                            adversaries, or adversaries that the precision of complex64 vectors cannot separate, show up
+                            here; u is still written */
 };
 
 #define DRACO_MAX_N 128  /* largest supported number of nodes */
 
 /* Device-side results of the most recent locate / decode on a plan. */
 typedef struct draco_info {
-    int32_t status;        /* DRACO_OK, DRACO_ETOOMANY or DRACO_ENOMAJ */
+    int32_t status;        /* DRACO_OK, DRACO_ETOOMANY, DRACO_ENOMAJ or DRACO_EUNSURE */
     int32_t n_flagged;     /* |V|: nodes flagged by the last locate (or given to the last cyclic decode) */
     int32_t locator_rank;  /* cyclic: numerical rank of the s x s syndrome system = adversaries seen */
     int32_t n_active;      /* cyclic decode: number of rows with b_j != 0 */
@@ -75,7 +81,9 @@ typedef struct draco_info {
     double max_syndrome;   /* cyclic: max_m |h_m| over the 2 s syndromes */
     int32_t internal_error; /* non-zero: a kernel gave up a bounded wait (sticky); draco_get_info then returns DRACO_EINTERNAL.
                                Always 0 with the current kernels, none of which spins on a flag */
-    int32_t reserved;
+    int32_t svd_sweeps;    /* cyclic locate: Jacobi sweeps the singular-value iteration of the s x s syndrome system took
+                              (0 when it was skipped: s = 0, or all syndromes within the cutoff); negative (minus the
+                              limit of 60) when it was still rotating at the limit: rank and V are then not to be trusted */
     double locator_margin; /* cyclic locate: |t| of the weakest flagged node / |t| of the strongest unflagged one (exactly
                               `rank` entries of t are non-zero in exact arithmetic, so this is large when the flags can be
                               trusted and near 1 when they cannot); 1e300 when no node or every node is flagged */
@@ -142,7 +150,10 @@ int draco_locate(draco_plan* plan, const void* R, const float* f, uint8_t* flags
  *               ascending, fp32; flags may be NULL and is ignored;
  *   cyclic:     Algorithm 1, steps 2-4: U = nodes with flags[j] = 0, b = the minimum-norm
  *               solution of W_{.,U} b = 1_P, u = Re(R_{.,U} b), fp64 accumulation, fp32 result.
- * flags: device [n] bytes (cyclic: required).  u: device [d] fp32.
+ * flags: device [n] bytes, or NULL.  Cyclic plans with flags == NULL decode with the set V that the most recent
+ * draco_locate / draco_cyc_locate_from_projection on this plan found (the plan keeps its own copy; no node is
+ * flagged on a plan that has not located yet), so locate and decode chain without the caller holding V.
+ * u: device [d] fp32.
  */
 int draco_decode(draco_plan* plan, const void* R, const uint8_t* flags, float* u, void* stream);
 

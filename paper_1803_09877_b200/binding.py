@@ -11,7 +11,7 @@ import os
 
 REP, CYC, CYC_PACKED = 0, 1, 2
 ADV_REVGRAD, ADV_CONST, ADV_GAUSS = 0, 1, 2
-OK, EINVAL, ECUDA, ETOOMANY, ENOMEM, EINTERNAL, ELIMIT, ENOMAJ = 0, -1, -2, -3, -4, -5, -6, 1
+OK, EINVAL, ECUDA, ETOOMANY, ENOMEM, EINTERNAL, ELIMIT, ENOMAJ, EUNSURE = 0, -1, -2, -3, -4, -5, -6, 1, 2
 MAX_N = 128
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -24,7 +24,7 @@ class DracoError(RuntimeError):
 class DracoInfo(C.Structure):
     _fields_ = [("status", C.c_int32), ("n_flagged", C.c_int32), ("locator_rank", C.c_int32),
                 ("n_active", C.c_int32), ("no_majority", C.c_uint64), ("scale", C.c_double),
-                ("max_syndrome", C.c_double), ("internal_error", C.c_int32), ("reserved", C.c_int32),
+                ("max_syndrome", C.c_double), ("internal_error", C.c_int32), ("svd_sweeps", C.c_int32),
                 ("locator_margin", C.c_double), ("im_residual", C.c_double), ("re_max", C.c_double)]
 
     def as_dict(self):

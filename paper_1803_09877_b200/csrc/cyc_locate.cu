@@ -45,15 +45,10 @@ __device__ __forceinline__ double cabs2(double2 a) { return a.x * a.x + a.y * a.
 // sqrt(s): at s = 20 that noise alone reached the rank cutoff and flagged an honest node.
 //
 // q_j = sum_i |R[j][i]|^2 travels with e_j: it is the yardstick of the locator's rank cutoff (rounding R to
-// complex64 perturbs e_j by about 2^-25 (E f^2 q_j)^(1/2), whatever e_j itself cancels to).  A few digits of it
-// are enough: fp32 terms and tile sums, fp64 across tiles.  Layout of the block partials: [grid][n] double2 (e),
-// then [grid][n] double (q).
-__device__ __forceinline__ float energy2(float4 v, float acc) {
-    acc = fmaf(v.x, v.x, acc);
-    acc = fmaf(v.y, v.y, acc);
-    acc = fmaf(v.z, v.z, acc);
-    return fmaf(v.w, v.w, acc);
-}
+// complex64 perturbs e_j by about 2^-25 (E f^2 q_j)^(1/2), whatever e_j itself cancels to).  It is summed in fp64
+// from the converted values as well: squares of fp32 values overflow fp32 from 1.8e19 on, which a node may well
+// send (W itself reaches 1e17 at n = 128, s = 20).  Layout of the block partials: [grid][n] double2 (e), then
+// [grid][n] double (q).
 __device__ __forceinline__ double warp_sum(double a) {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
@@ -99,7 +94,7 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
             const int j = row0 + warp + r * kProjectWarps;
             if (j < row0 + nrows) {
                 const float2* row = R + (int64_t)j * ld + c0;
-                float eq = 0.f;
+                double eq = 0.0;
                 double ar = 0.0, ai = 0.0;
                 if (VEC2 && cnt == kProjectTile) {
                     const float4* row4 = reinterpret_cast<const float4*>(row);
@@ -108,29 +103,29 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
                         float4 v[8];
 #pragma unroll
                         for (int q = 0; q < 8; ++q) v[q] = __ldcs(row4 + (step0 + q) * 32 + lane);
-                        float pq = 0.f;
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
                             const double2 ff = *reinterpret_cast<const double2*>(&fs[((step0 + q) * 32 + lane) * 2]);
-                            ar = fma(ff.x, (double)v[q].x, ar); ai = fma(ff.x, (double)v[q].y, ai);
-                            ar = fma(ff.y, (double)v[q].z, ar); ai = fma(ff.y, (double)v[q].w, ai);
-                            pq = energy2(v[q], pq);
+                            const double x0 = (double)v[q].x, y0 = (double)v[q].y, x1 = (double)v[q].z, y1 = (double)v[q].w;
+                            ar = fma(ff.x, x0, ar); ai = fma(ff.x, y0, ai);
+                            ar = fma(ff.y, x1, ar); ai = fma(ff.y, y1, ai);
+                            eq = fma(x0, x0, eq); eq = fma(y0, y0, eq);
+                            eq = fma(x1, x1, eq); eq = fma(y1, y1, eq);
                         }
-                        eq += pq;
                     }
                 } else {
                     for (int i = lane; i < cnt; i += 32) {
                         const float2 v = __ldcs(row + i);
-                        const double ff = fs[i];
-                        ar = fma(ff, (double)v.x, ar);
-                        ai = fma(ff, (double)v.y, ai);
-                        eq = fmaf(v.y, v.y, fmaf(v.x, v.x, eq));
+                        const double ff = fs[i], x0 = (double)v.x, y0 = (double)v.y;
+                        ar = fma(ff, x0, ar);
+                        ai = fma(ff, y0, ai);
+                        eq = fma(y0, y0, fma(x0, x0, eq));
                     }
                 }
                 accr[r] += ar;
                 acci[r] += ai;
                 eq = warp_sum(eq);
-                if (lane == 0) qs[r * kProjectWarps + warp] += (double)eq;
+                if (lane == 0) qs[r * kProjectWarps + warp] += eq;
             }
         }
         __syncthreads();
@@ -169,9 +164,10 @@ cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict
     __shared__ double wq[kProjectWarps][NMAX];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     double accr[NMAX], acci[NMAX];
-    float accq[NMAX];                                    // q needs a few digits only: fp32 running sums
 #pragma unroll
-    for (int j = 0; j < NMAX; ++j) { accr[j] = 0.0; acci[j] = 0.0; accq[j] = 0.f; }
+    for (int j = 0; j < NMAX; ++j) { accr[j] = 0.0; acci[j] = 0.0; }
+    if (lane < NMAX) wq[warp][lane] = 0.0;               // q_j of this warp's chunks: summed over the lanes per chunk, kept here
+    __syncwarp();
     const int64_t nchunks = (len + CH - 1) / CH;
     const int64_t nwarps = (int64_t)gridDim.x * kProjectWarps;
     for (int64_t chunk = (int64_t)blockIdx.x * kProjectWarps + warp; chunk < nchunks; chunk += nwarps) {
@@ -194,30 +190,40 @@ cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict
 #pragma unroll
                         for (int q = 0; q < 4; ++q) vb[q] = __ldcs(rb + q * 32 + lane);
                     }
+                    double qa = 0.0, qb = 0.0;
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const double fx = (double)ff[q].x, fy = (double)ff[q].y;     // shared by the two rows
-                        accr[jj] = fma(fx, (double)va[q].x, accr[jj]); acci[jj] = fma(fx, (double)va[q].y, acci[jj]);
-                        accr[jj] = fma(fy, (double)va[q].z, accr[jj]); acci[jj] = fma(fy, (double)va[q].w, acci[jj]);
-                        accq[jj] = energy2(va[q], accq[jj]);
+                        double x0 = (double)va[q].x, y0 = (double)va[q].y, x1 = (double)va[q].z, y1 = (double)va[q].w;
+                        accr[jj] = fma(fx, x0, accr[jj]); acci[jj] = fma(fx, y0, acci[jj]);
+                        accr[jj] = fma(fy, x1, accr[jj]); acci[jj] = fma(fy, y1, acci[jj]);
+                        qa = fma(x0, x0, qa); qa = fma(y0, y0, qa); qa = fma(x1, x1, qa); qa = fma(y1, y1, qa);
                         if (two) {
-                            accr[jj + 1] = fma(fx, (double)vb[q].x, accr[jj + 1]); acci[jj + 1] = fma(fx, (double)vb[q].y, acci[jj + 1]);
-                            accr[jj + 1] = fma(fy, (double)vb[q].z, accr[jj + 1]); acci[jj + 1] = fma(fy, (double)vb[q].w, acci[jj + 1]);
-                            accq[jj + 1] = energy2(vb[q], accq[jj + 1]);
+                            x0 = (double)vb[q].x; y0 = (double)vb[q].y; x1 = (double)vb[q].z; y1 = (double)vb[q].w;
+                            accr[jj + 1] = fma(fx, x0, accr[jj + 1]); acci[jj + 1] = fma(fx, y0, acci[jj + 1]);
+                            accr[jj + 1] = fma(fy, x1, accr[jj + 1]); acci[jj + 1] = fma(fy, y1, acci[jj + 1]);
+                            qb = fma(x0, x0, qb); qb = fma(y0, y0, qb); qb = fma(x1, x1, qb); qb = fma(y1, y1, qb);
                         }
                     }
+                    qa = warp_sum(qa);
+                    qb = warp_sum(qb);
+                    if (lane == 0) { wq[warp][jj] += qa; if (two) wq[warp][jj + 1] += qb; }
                 }
             }
         } else {
-            for (int i = lane; i < cnt; i += 32) {
-                const double fi = (double)__ldcs(f + c0 + i);
+            for (int i0 = 0; i0 < cnt; i0 += 32) {           // every lane takes part in the sums over the lanes below
+                const int i = i0 + lane;
+                const bool valid = i < cnt;
+                const double fi = valid ? (double)__ldcs(f + c0 + i) : 0.0;
 #pragma unroll
                 for (int j = 0; j < NMAX; ++j)
                     if (j < n) {
-                        const float2 v = __ldcs(R + (int64_t)j * ld + c0 + i);
-                        accr[j] = fma(fi, (double)v.x, accr[j]);
-                        acci[j] = fma(fi, (double)v.y, acci[j]);
-                        accq[j] = fmaf(v.y, v.y, fmaf(v.x, v.x, accq[j]));
+                        const float2 v = valid ? __ldcs(R + (int64_t)j * ld + c0 + i) : make_float2(0.f, 0.f);
+                        const double x0 = (double)v.x, y0 = (double)v.y;
+                        accr[j] = fma(fi, x0, accr[j]);
+                        acci[j] = fma(fi, y0, acci[j]);
+                        const double qv = warp_sum(fma(y0, y0, x0 * x0));
+                        if (lane == 0) wq[warp][j] += qv;
                     }
             }
         }
@@ -230,8 +236,7 @@ cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict
             a += __shfl_xor_sync(0xffffffffu, a, off);
             b += __shfl_xor_sync(0xffffffffu, b, off);
         }
-        const double c = warp_sum((double)accq[j]);
-        if (lane == 0) { wsum[warp][j] = make_double2(a, b); wq[warp][j] = c; }
+        if (lane == 0) wsum[warp][j] = make_double2(a, b);
     }
     __syncthreads();
     if (threadIdx.x < n) {
@@ -411,7 +416,9 @@ __device__ int block_jacobi_pinv(double2* A, double2* V, const double2* rhs, int
         V[idx] = make_double2(c == i ? 1.0 : 0.0, 0.0);
     }
     __syncthreads();
-    for (int sweep = 0; sweep < 60; ++sweep) {
+    int sweeps = 0;
+    bool converged = false;
+    for (int sweep = 0; sweep < kJacobiSweepLimit; ++sweep) {
         if (tid == 0) sh[0] = 0;
         __syncthreads();
         for (int step = 0; step < sp - 1; ++step) {
@@ -454,9 +461,10 @@ __device__ int block_jacobi_pinv(double2* A, double2* V, const double2* rhs, int
         }
         const int rotated = sh[0];
         __syncthreads();
-        if (!rotated) break;
+        ++sweeps;
+        if (!rotated) { converged = true; break; }
     }
-    if (tid == 0) sh[1] = 0;
+    if (tid == 0) { sh[1] = 0; sh[3] = converged ? sweeps : -sweeps; }
     __syncthreads();
     if (tid < sp) {
         const double2* ak = A + tid * sp;
@@ -504,7 +512,9 @@ __device__ int warp_jacobi_pinv(double2* A, double2* V, const double2* rhs, int 
         V[idx] = make_double2(c == i ? 1.0 : 0.0, 0.0);
     }
     __syncwarp();
-    for (int sweep = 0; sweep < 60; ++sweep) {
+    int sweeps = 0;
+    bool converged = false;
+    for (int sweep = 0; sweep < kJacobiSweepLimit; ++sweep) {
         bool rotated = false;
         for (int step = 0; step < sp - 1; ++step) {
             int p = 0, q = 1;
@@ -553,7 +563,8 @@ __device__ int warp_jacobi_pinv(double2* A, double2* V, const double2* rhs, int 
             }
             __syncwarp();
         }
-        if (!__any_sync(full, rotated)) break;
+        ++sweeps;
+        if (!__any_sync(full, rotated)) { converged = true; break; }
     }
     bool keep = false;
     if (lane < sp) {
@@ -579,7 +590,7 @@ __device__ int warp_jacobi_pinv(double2* A, double2* V, const double2* rhs, int 
         }
         beta[lane] = make_double2(re, im);
     }
-    if (lane == 0) sh[1] = rank;
+    if (lane == 0) { sh[1] = rank; sh[3] = converged ? sweeps : -sweeps; }
     __syncwarp();
     return rank;
 }
@@ -610,7 +621,7 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, int n, int s, 
         mag[tid] = sqrt(qv[tid]);
         h[tid] = make_double2(0.0, 0.0);
     }
-    if (tid == 0) count = 0;
+    if (tid == 0) { count = 0; sh[3] = 0; }
     __syncthreads();
     // scale = median of q_j^(1/2) by rank counting
     if (tid < n) {
@@ -729,9 +740,14 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, int n, int s, 
         info->locator_rank = rank;
         info->scale = scale_s;
         info->max_syndrome = maxsyn_s;
-        info->status = DRACO_OK;
+        const double margin = (rank > 0 && rank < n) ? sqrt(sorted[0] / fmax(sorted[1], 1e-300)) : 1e300;
+        // exactly `rank` entries of t are non-zero in exact arithmetic: where the weakest flagged and the strongest
+        // unflagged |t_j| are less than a decade apart the choice of V is not to be trusted, nor is a rank that comes
+        // from an iteration that was stopped at its sweep limit (NaN in R makes the comparison false: unsure)
+        info->status = (margin >= kMarginBar && sh[3] >= 0) ? DRACO_OK : DRACO_EUNSURE;
         info->no_majority = 0;
-        info->locator_margin = (rank > 0 && rank < n) ? sqrt(sorted[0] / fmax(sorted[1], 1e-300)) : 1e300;
+        info->locator_margin = margin;
+        info->svd_sweeps = sh[3];
     }
 }
 

@@ -245,7 +245,7 @@ int draco_cyc_locate_from_projection(draco_plan* plan, const double* e, uint8_t*
 }
 
 int draco_locate(draco_plan* plan, const void* R, const float* f, uint8_t* flags, void* stream) {
-    if (!plan || !R || !flags || !aligned16(R)) return DRACO_EINVAL;
+    if (!plan || !R || !aligned16(R)) return DRACO_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     if (plan->code == DRACO_REP)
         return launch_rep_vote(plan, (const float*)R, plan->d, plan->d, nullptr, nullptr, flags, true, st);
@@ -260,7 +260,7 @@ int draco_decode(draco_plan* plan, const void* R, const uint8_t* flags, float* u
     cudaStream_t st = (cudaStream_t)stream;
     if (plan->code == DRACO_REP)
         return launch_rep_vote(plan, (const float*)R, plan->d, plan->d, u, nullptr, nullptr, true, st);
-    if (!flags) return DRACO_EINVAL;
+    if (!flags) flags = plan->flags_dev;                 // the plan's own copy of its last locate's flags
     int rc = launch_cyc_decode_vector(plan, flags, st);
     if (rc != DRACO_OK) return rc;
     return launch_cyc_recover(plan, (const float2*)R, vec_len(plan), vec_len(plan), u, is_packed(plan) ? plan->d : 0, st);
@@ -271,7 +271,7 @@ int draco_decode_update(draco_plan* plan, const void* R, const uint8_t* flags, f
     cudaStream_t st = (cudaStream_t)stream;
     if (plan->code == DRACO_REP)
         return launch_rep_vote(plan, (const float*)R, plan->d, plan->d, nullptr, nullptr, nullptr, true, st, w, scale);
-    if (!flags) return DRACO_EINVAL;
+    if (!flags) flags = plan->flags_dev;
     int rc = launch_cyc_decode_vector(plan, flags, st);
     if (rc != DRACO_OK) return rc;
     return launch_cyc_recover(plan, (const float2*)R, vec_len(plan), vec_len(plan), nullptr, is_packed(plan) ? plan->d : 0, st, w,
@@ -310,10 +310,15 @@ int draco_get_info(draco_plan* plan, draco_info* info, void* stream) {
     info->scale = h.scale;
     info->max_syndrome = h.max_syndrome;
     info->internal_error = h.internal_error;
-    info->reserved = 0;
+    info->svd_sweeps = h.svd_sweeps;
     info->locator_margin = h.locator_margin;
     memcpy(&info->im_residual, &h.im_residual_bits, sizeof(double));
     memcpy(&info->re_max, &h.re_max_bits, sizeof(double));
+    // The recovery kernel's blocks only merge their maxima; the verdict on them is formed here.  u-hat = G 1_P is
+    // real: an imaginary part beyond rounding means an adversary is still among the rows that were combined.
+    // (NaN from an adversary compares false with everything and so counts as a failed check.)
+    if (is_cyc(plan) && info->status == DRACO_OK && !(info->im_residual <= kImResidualBar * info->re_max))
+        info->status = DRACO_EUNSURE;
     return h.internal_error ? DRACO_EINTERNAL : DRACO_OK;
 }
 
@@ -439,6 +444,7 @@ const char* draco_strerror(int code) {
         case DRACO_EINTERNAL: return "a bounded wait inside a kernel expired";
         case DRACO_ELIMIT: return "size exceeds a fixed capacity of this entry point";
         case DRACO_ENOMAJ: return "no strict majority at some coordinate";
+        case DRACO_EUNSURE: return "a self-check of the cyclic decoder failed: the flags or the sum may be wrong";
         default: return "unknown code";
     }
 }

@@ -12,6 +12,9 @@ constexpr int kMaxN = DRACO_MAX_N;
 constexpr int kMaxTaps = 15;          // 2 s + 1 for the register-window encoder (s <= 7)
 constexpr int kProjectTile = 2048;    // coordinates per tile of the projection kernel
 constexpr int kProjectWarps = 8;
+constexpr double kMarginBar = 10.0;        // locator_margin below this, or ..
+constexpr double kImResidualBar = 1e-2;    // .. im_residual above this fraction of re_max: status DRACO_EUNSURE
+constexpr int kJacobiSweepLimit = 60;
 
 struct GroupTable {                   // repetition code: consecutive groups
     int num_groups;
@@ -60,7 +63,7 @@ struct DeviceInfo {                   // mirrors draco_info
     double scale;
     double max_syndrome;
     int32_t internal_error;
-    int32_t reserved;
+    int32_t svd_sweeps;
     double locator_margin;
     unsigned long long im_residual_bits;   // bit patterns of non-negative doubles: they order like integers, so the
     unsigned long long re_max_bits;        // blocks of the recovery kernel merge their maxima with atomicMax

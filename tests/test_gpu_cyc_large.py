@@ -67,6 +67,9 @@ def _check_locate_decode(dr, n, s, d, n_adv, model, packed, seed=None):
     assert np.abs(eg[: 2 * n].view(np.complex128) - want["e"]).max() <= 1e-6 * np.abs(want["e"]).max()
     qo = orc.cyc_project_energy(R)
     assert np.abs(eg[2 * n:] - qo).max() <= 1e-5 * qo.max()
+    # exact products, fp64 sums: only the order of the additions differs from the oracle's
+    assert np.abs(eg[: 2 * n].view(np.complex128) - want["e"]).max() <= 1e-11 * np.sqrt(qo.max() * 2 * vlen)
+    assert np.abs(eg[2 * n:] - qo).max() <= 1e-12 * qo.max()
     # flags and rank
     # The singular values that stand for "zero" are rounding noise.  Both sides see the noise of the complex64
     # vectors; the device adds that of its fp32 products, of the same size, so its noise may be sqrt(2) times
@@ -86,7 +89,11 @@ def _check_locate_decode(dr, n, s, d, n_adv, model, packed, seed=None):
     u = torch.full((d,), float("nan"), dtype=torch.float32, device="cuda")
     plan.decode(Rd, flags, u)
     info = plan.info()
-    assert info["status"] == 0 and info["n_active"] == n - n_adv
+    assert info["n_active"] == n - n_adv
+    # where the code's cancellation leaves nothing of the sum (its imaginary part is as large as its real part)
+    # the decoder says so; otherwise the status is clean
+    unsure = (not packed) and not (info["im_residual"] <= 1e-2 * info["re_max"])
+    assert info["status"] == (dr.binding.EUNSURE if unsure else 0)
     b, bo = plan.cyc_decode_vector(), orc.cyc_decode_vector(n, s, want["flags"])
     db = float(np.abs(b - bo).max() / np.abs(bo).max())
     assert db <= _b_bar(n, s, want["flags"])[1]
@@ -156,7 +163,8 @@ def test_decode_vector_with_more_than_16_flags(n, s, d, n_flags):
     u = torch.full((d,), float("nan"), dtype=torch.float32, device="cuda")
     plan.decode(dev(R), dev(flags), u)
     info = plan.info()
-    assert info["status"] == 0 and info["n_active"] == n - k and info["n_flagged"] == k
+    # R is random, not a set of coded vectors: u-hat comes out as complex as it is real, which the self-check reports
+    assert info["status"] == dr.binding.EUNSURE and info["n_active"] == n - k and info["n_flagged"] == k
     b, bo = plan.cyc_decode_vector(), orc.cyc_decode_vector(n, s, flags.astype(bool))
     assert not np.abs(b[flags.astype(bool)]).any()
     db = float(np.abs(b - bo).max() / np.abs(bo).max())
