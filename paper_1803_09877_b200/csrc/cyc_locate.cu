@@ -73,14 +73,18 @@ __global__ void __launch_bounds__(kThreads, 4)
 cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
                    int row0, int nrows, double2* __restrict__ partial, int accumulate) {
     __shared__ __align__(16) double fs[kProjectTile];
-    __shared__ double qs[kProjectWarps * RPW];           // q of row warp + r * 8, kept by lane 0 of its warp
+    // Running sums of row warp + r * 8 over this block's tiles, kept by lane 0 of the row's warp: after every tile
+    // the warp adds its lanes' sums up (fixed butterfly order) and lane 0 adds the result here.  Keeping them in
+    // registers instead (2 RPW doubles per lane) left too few of the 64 registers for eight 128-bit loads in flight.
+    __shared__ double2 es[kProjectWarps * RPW];
+    __shared__ double qs[kProjectWarps * RPW];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    double accr[RPW], acci[RPW];
-#pragma unroll
-    for (int r = 0; r < RPW; ++r) { accr[r] = 0.0; acci[r] = 0.0; }
     if (lane == 0) {
 #pragma unroll
-        for (int r = 0; r < RPW; ++r) qs[r * kProjectWarps + warp] = 0.0;
+        for (int r = 0; r < RPW; ++r) {
+            es[r * kProjectWarps + warp] = make_double2(0.0, 0.0);
+            qs[r * kProjectWarps + warp] = 0.0;
+        }
     }
 
     const int64_t ntiles = (len + kProjectTile - 1) / kProjectTile;
@@ -122,31 +126,34 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
                         eq = fma(y0, y0, fma(x0, x0, eq));
                     }
                 }
-                accr[r] += ar;
-                acci[r] += ai;
+                ar = warp_sum(ar);
+                ai = warp_sum(ai);
                 eq = warp_sum(eq);
-                if (lane == 0) qs[r * kProjectWarps + warp] += eq;
+                if (lane == 0) {
+                    double2 acc = es[r * kProjectWarps + warp];
+                    acc.x += ar;
+                    acc.y += ai;
+                    es[r * kProjectWarps + warp] = acc;
+                    qs[r * kProjectWarps + warp] += eq;
+                }
             }
         }
         __syncthreads();
     }
     double* qpartial = q_partials(partial, n);
+    if (lane == 0) {
 #pragma unroll
-    for (int r = 0; r < RPW; ++r) {
-        double a = accr[r], b = acci[r];
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            a += __shfl_xor_sync(0xffffffffu, a, off);
-            b += __shfl_xor_sync(0xffffffffu, b, off);
-        }
-        const int j = row0 + warp + r * kProjectWarps;
-        if (lane == 0 && j < row0 + nrows) {
-            double2* dst = partial + (int64_t)blockIdx.x * n + j;
-            double* qdst = qpartial + (int64_t)blockIdx.x * n + j;
-            double c = qs[r * kProjectWarps + warp];
-            if (accumulate) { a += dst->x; b += dst->y; c += *qdst; }
-            *dst = make_double2(a, b);
-            *qdst = c;
+        for (int r = 0; r < RPW; ++r) {
+            const int j = row0 + warp + r * kProjectWarps;
+            if (j < row0 + nrows) {
+                double2* dst = partial + (int64_t)blockIdx.x * n + j;
+                double* qdst = qpartial + (int64_t)blockIdx.x * n + j;
+                double2 a = es[r * kProjectWarps + warp];
+                double c = qs[r * kProjectWarps + warp];
+                if (accumulate) { a.x += dst->x; a.y += dst->y; c += *qdst; }
+                *dst = a;
+                *qdst = c;
+            }
         }
     }
 }
