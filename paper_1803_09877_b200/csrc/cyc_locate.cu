@@ -59,8 +59,10 @@ __device__ __forceinline__ float warp_sum(float a) {
     for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
     return a;
 }
-__device__ __forceinline__ double* q_partials(double2* partial, int n) {
-    return reinterpret_cast<double*>(partial + (int64_t)gridDim.x * n);
+// Block partials: [cap][n] double2 (e) followed by [cap][n] double (q); cap = the capacity of the buffer in blocks,
+// of which a launch fills the first gridDim.x.
+__device__ __forceinline__ double* q_partials(double2* partial, int cap, int n) {
+    return reinterpret_cast<double*>(partial + (int64_t)cap * n);
 }
 // Block = 8 warps over one tile of coordinates; warp w owns rows row0 + w, row0 + w + 8, ... of the
 // launch's nrows <= 8 RPW rows; f for the tile sits in shared memory as fp64 (converted once per tile, used by
@@ -71,7 +73,7 @@ __device__ __forceinline__ double* q_partials(double2* partial, int n) {
 template <int RPW, bool VEC2>
 __global__ void __launch_bounds__(kThreads, 4)
 cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
-                   int row0, int nrows, double2* __restrict__ partial, int accumulate) {
+                   int row0, int nrows, double2* __restrict__ partial, int cap, int accumulate) {
     __shared__ __align__(16) double fs[kProjectTile];
     // Running sums of row warp + r * 8 over this block's tiles, kept by lane 0 of the row's warp: after every tile
     // the warp adds its lanes' sums up (fixed butterfly order) and lane 0 adds the result here.  Keeping them in
@@ -140,7 +142,7 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
         }
         __syncthreads();
     }
-    double* qpartial = q_partials(partial, n);
+    double* qpartial = q_partials(partial, cap, n);
     if (lane == 0) {
 #pragma unroll
         for (int r = 0; r < RPW; ++r) {
@@ -165,7 +167,7 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
 template <bool VEC2>
 __global__ void __launch_bounds__(kThreads, 2)
 cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict__ f, int64_t len, int64_t ld, int n,
-                           double2* __restrict__ partial, int accumulate) {
+                           double2* __restrict__ partial, int cap, int accumulate) {
     constexpr int NMAX = 16, CH = 256;
     __shared__ double2 wsum[kProjectWarps][NMAX];
     __shared__ double wq[kProjectWarps][NMAX];
@@ -254,7 +256,7 @@ cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict
             c += wq[w][threadIdx.x];
         }
         double2* dst = partial + (int64_t)blockIdx.x * n + threadIdx.x;
-        double* qdst = q_partials(partial, n) + (int64_t)blockIdx.x * n + threadIdx.x;
+        double* qdst = q_partials(partial, cap, n) + (int64_t)blockIdx.x * n + threadIdx.x;
         if (accumulate) { a += dst->x; b += dst->y; c += *qdst; }
         *dst = make_double2(a, b);
         *qdst = c;
@@ -268,11 +270,11 @@ cyc_project_fewrows_kernel(const float2* __restrict__ R, const float* __restrict
 // 20-40 us: one SM's load latency, serialised.)
 constexpr int kReduceThreads = 128;
 __global__ void __launch_bounds__(kReduceThreads)
-cyc_reduce_partials_kernel(const double2* __restrict__ partial, int grid, int n, double* __restrict__ record) {
+cyc_reduce_partials_kernel(const double2* __restrict__ partial, int grid, int cap, int n, double* __restrict__ record) {
     constexpr int kBatch = 8;
     __shared__ double wsum[3][kReduceThreads / 32];
     const int j = blockIdx.x, tid = threadIdx.x;
-    const double* __restrict__ qpartial = reinterpret_cast<const double*>(partial + (int64_t)grid * n);
+    const double* __restrict__ qpartial = reinterpret_cast<const double*>(partial + (int64_t)cap * n);
     double a = 0.0, b = 0.0, c = 0.0;
     for (int base = 0; base < grid; base += kBatch * kReduceThreads) {
         double2 pe[kBatch];
@@ -389,20 +391,31 @@ __device__ int block_gauss_jordan(double2* A, int dim, double tol, double2* x, i
     return rank;
 }
 
-// Rotation of one Jacobi pair from alpha = |a_p|^2, beta = |a_q|^2 and gamma = a_p^H a_q (g2 = |gamma|^2 > 0):
-// ph = exp(-i arg gamma), t = sign(zeta) / (|zeta| + sqrt(1 + zeta^2)) with zeta = (beta - alpha) / (2 |gamma|),
-// c = 1 / sqrt(1 + t^2), s = c t.  Written with four long-latency operations (two reciprocal square roots, a
-// square root and a division) instead of seven: t = sign(delta) 2 |gamma| / (|delta| + sqrt(delta^2 + 4 |gamma|^2)),
-// delta = beta - alpha.  The chain is serial and is most of a Jacobi step.
-__device__ __forceinline__ void jacobi_rotation(double alpha, double bet, double gr, double gi, double g2, double2& ph,
-                                                double& c, double& sn) {
-    const double rg = rsqrt(g2);
-    const double g = g2 * rg;
-    ph = make_double2(gr * rg, -gi * rg);
+// Rotation of one Jacobi pair from alpha = |a_p|^2, beta = |a_q|^2 and gamma = a_p^H a_q (g2 = |gamma|^2 > 0): the
+// unitary [[c, st], [-conj(st), c]] (c real, st complex) that makes the new columns a_p' = c a_p - conj(st) a_q and
+// a_q' = st a_p + c a_q orthogonal, the smaller of the two angles.  With delta = beta - alpha, h = (delta^2 +
+// 4 |gamma|^2)^(1/2) and x = |delta| / h:  c^2 = (1 + x) / 2,  st = sign(delta) gamma / (h c).  (The textbook form
+// first turns a_q by exp(-i arg gamma) and then rotates by a real angle; the result differs by a unit factor on the
+// second column, which one-sided Jacobi does not care about.)  Two reciprocal square roots and no division or square
+// root: the chain of long-latency operations is serial and is most of a Jacobi step.
+__device__ __forceinline__ void jacobi_rotation(double alpha, double bet, double gr, double gi, double g2, double& c,
+                                                double2& st) {
     const double delta = bet - alpha;
-    const double tt = copysign(2.0 * g, delta) / (fabs(delta) + sqrt(fma(delta, delta, 4.0 * g2)));
-    c = rsqrt(fma(tt, tt, 1.0));
-    sn = c * tt;
+    const double rh = rsqrt(fma(delta, delta, 4.0 * g2));
+    const double c2 = fma(0.5 * fabs(delta), rh, 0.5);
+    const double rc = rsqrt(c2);
+    c = c2 * rc;
+    const double k = copysign(rh * rc, delta);
+    st = make_double2(gr * k, gi * k);
+}
+
+// one column pair, rows i0, i0 + step, ..: (x, y) <- (c x - conj(st) y, st x + c y)
+__device__ __forceinline__ void rotate_pair(double2* xp, double2* yp, int i0, int step, int rows, double c, double2 st) {
+    for (int i = i0; i < rows; i += step) {
+        const double2 x = xp[i], y = yp[i];
+        xp[i] = make_double2(c * x.x - (st.x * y.x + st.y * y.y), c * x.y - (st.x * y.y - st.y * y.x));
+        yp[i] = make_double2(st.x * x.x - st.y * x.y + c * y.x, st.x * x.y + st.y * x.x + c * y.y);
+    }
 }
 
 // ------------------------------------------------------------------ small SVD solve
@@ -446,21 +459,11 @@ __device__ int block_jacobi_pinv(double2* A, double2* V, const double2* rhs, int
                 }
                 const double g2 = gr * gr + gi * gi;
                 if (g2 > 1e-30 * alpha * bet && g2 > 0.0) {
-                    double2 ph;
-                    double c, sn;
-                    jacobi_rotation(alpha, bet, gr, gi, g2, ph, c, sn);
-                    for (int i = 0; i < s; ++i) {
-                        const double2 x = ap[i], y = cmul(aq[i], ph);
-                        ap[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
-                        aq[i] = make_double2(sn * x.x + c * y.x, sn * x.y + c * y.y);
-                    }
-                    double2* vp = V + p * sp;
-                    double2* vq = V + q * sp;
-                    for (int i = 0; i < sp; ++i) {
-                        const double2 x = vp[i], y = cmul(vq[i], ph);
-                        vp[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
-                        vq[i] = make_double2(sn * x.x + c * y.x, sn * x.y + c * y.y);
-                    }
+                    double c;
+                    double2 st;
+                    jacobi_rotation(alpha, bet, gr, gi, g2, c, st);
+                    rotate_pair(ap, aq, 0, 1, s, c, st);
+                    rotate_pair(V + p * sp, V + q * sp, 0, 1, sp, c, st);
                     sh[0] = 1;
                 }
             }
@@ -551,21 +554,11 @@ __device__ int warp_jacobi_pinv(double2* A, double2* V, const double2* rhs, int 
             }
             const double g2 = gr * gr + gi * gi;
             if (act && g2 > 1e-30 * alpha * bet && g2 > 0.0) {
-                double2 ph;
-                double c, sn;
-                jacobi_rotation(alpha, bet, gr, gi, g2, ph, c, sn);
-                for (int i = sub; i < s; i += lp) {
-                    const double2 x = ap[i], y = cmul(aq[i], ph);
-                    ap[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
-                    aq[i] = make_double2(sn * x.x + c * y.x, sn * x.y + c * y.y);
-                }
-                double2* vp = V + p * sp;
-                double2* vq = V + q * sp;
-                for (int i = sub; i < sp; i += lp) {
-                    const double2 x = vp[i], y = cmul(vq[i], ph);
-                    vp[i] = make_double2(c * x.x - sn * y.x, c * x.y - sn * y.y);
-                    vq[i] = make_double2(sn * x.x + c * y.x, sn * x.y + c * y.y);
-                }
+                double c;
+                double2 st;
+                jacobi_rotation(alpha, bet, gr, gi, g2, c, st);
+                rotate_pair(ap, aq, sub, lp, s, c, st);
+                rotate_pair(V + p * sp, V + q * sp, sub, lp, sp, c, st);
                 rotated = true;
             }
             __syncwarp();
@@ -603,11 +596,132 @@ __device__ int warp_jacobi_pinv(double2* A, double2* V, const double2* rhs, int 
 }
 
 constexpr int kSmallDim = 16;         // systems up to this size are solved in shared memory by one warp
+constexpr int kFusedReduceMax = 64;   // up to this many block partials are added up by the locator kernel itself
+
+// ------------------------------------------------------------------ decode vector
+// With B = [C_L]_{.,V} and A = [C_L]_{.,U}: A A^H = I - B B^H, so the minimum-norm solution of
+// A b_U = e_last is b_U = A^H y, y = e_last + B (I - B^H B)^{-1} B^H e_last, and
+// I - B^H B = [C_R]_{.,V}^H [C_R]_{.,V} is only |V| x |V| (|V| <= 2 s).
+// Called by every thread of a block of kSolveThreads threads; flags may point to global or to shared memory.
+__device__ void decode_vector_body(CycDevice* cd, const uint8_t* flags, int n, int s, DeviceInfo* info) {
+    __shared__ int vlist[kMaxN], rowbestc[kMaxN], perm_s[kMaxN], sh[4], a_s;
+    __shared__ uint8_t fl[kMaxN];
+    __shared__ double rowbest[kMaxN];
+    __shared__ double2 y[kMaxN], tw[kMaxN], x_s[kMaxN], b_s[kMaxN];
+    __shared__ double2 As[kSmallDim * (kSmallDim + 1)];
+    const int tid = threadIdx.x;
+    const int rows = n - 2 * s, L = rows - 1;
+    const double rsn = 1.0 / sqrt((double)n);
+    if (tid < n) {
+        tw[tid] = cd->twiddle[tid];
+        fl[tid] = flags[tid];
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int a = 0;
+        for (int j = 0; j < n; ++j)
+            if (fl[j]) vlist[a++] = j;
+        a_s = a;
+    }
+    __syncthreads();
+    const int a = a_s;
+    if (a > 2 * s) {                                       // fewer than n - 2 s rows left: no b exists
+        if (tid < n) cd->b[tid] = make_double2(0.0, 0.0);
+        if (tid == 0) {
+            info->n_active = 0; info->n_flagged = a; info->status = DRACO_ETOOMANY;
+            info->im_residual_bits = 0ull; info->re_max_bits = 0ull;
+        }
+        return;
+    }
+    double2* x = x_s;
+    if (a > 0) {
+        const bool small = a <= kSmallDim;
+        double2* A = small ? As : cd->work;
+        for (int idx = tid; idx < a * (a + 1); idx += blockDim.x) {
+            const int p = idx / (a + 1), q = idx % (a + 1);
+            double2 val;
+            if (q < a) {                                   // (1/n) sum_{m >= n-2s} w^(m (v_q - v_p))
+                int dv = vlist[q] - vlist[p];
+                if (dv < 0) dv += n;
+                double re = 0.0, im = 0.0;
+                int k = ((n - 2 * s) * dv) % n;
+                for (int m = n - 2 * s; m < n; ++m) {
+                    const double2 w = tw[k];
+                    re += w.x;
+                    im += w.y;
+                    k += dv;
+                    if (k >= n) k -= n;
+                }
+                val = make_double2(re / n, im / n);
+            } else {                                       // conj(C[L][v_p])
+                const double2 w = tw[(L * vlist[p]) % n];
+                val = make_double2(w.x * rsn, -w.y * rsn);
+            }
+            A[idx] = val;
+        }
+        __syncthreads();
+        if (small) {
+            if (tid < 32) block_gauss_jordan<true>(A, a, 0.0, x, perm_s, rowbest, rowbestc, sh);
+            __syncthreads();
+        } else {
+            block_gauss_jordan<false>(A, a, 0.0, x, perm_s, rowbest, rowbestc, sh);
+        }
+    }
+    if (tid < rows) {
+        double re = (tid == L) ? 1.0 : 0.0, im = 0.0;
+        for (int p = 0; p < a; ++p) {
+            const double2 w = tw[(tid * vlist[p]) % n];
+            const double2 q = cmul(w, x[p]);
+            re += q.x * rsn;
+            im += q.y * rsn;
+        }
+        y[tid] = make_double2(re, im);
+    }
+    __syncthreads();
+    if (tid < n) {
+        double2 b = make_double2(0.0, 0.0);
+        if (!fl[tid]) {
+            double re = 0.0, im = 0.0;
+            int k = 0;                                     // (m tid) mod n
+            for (int m = 0; m < rows; ++m) {
+                const double2 q = cmulc(y[m], tw[k]);
+                re += q.x;
+                im += q.y;
+                k += tid;
+                if (k >= n) k -= n;
+            }
+            b = make_double2(re * rsn, im * rsn);
+        }
+        cd->b[tid] = b;
+        b_s[tid] = b;
+    }
+    __syncthreads();
+    // the active rows in ascending order: position = number of unflagged nodes before this one
+    if (tid < n && !fl[tid]) {
+        int k = 0;
+        for (int j = 0; j < tid; ++j) k += fl[j] ? 0 : 1;
+        cd->active[k] = tid;
+        cd->b_active[k] = b_s[tid];
+    }
+    if (tid == 0) {
+        info->n_active = n - a;
+        info->n_flagged = a;
+        info->im_residual_bits = 0ull;                     // the recovery kernel's blocks merge their maxima into these
+        info->re_max_bits = 0ull;
+        if (info->status == DRACO_ETOOMANY) info->status = DRACO_OK;
+    }
+}
+
+
+__global__ void __launch_bounds__(kSolveThreads)
+cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n, int s, DeviceInfo* info) {
+    decode_vector_body(cd, flags, n, s, info);
+}
 
 // ------------------------------------------------------------------ locator after the projection
 __global__ void __launch_bounds__(kSolveThreads)
-cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, int n, int s, double theta, uint8_t* flags,
-                 uint8_t* flags2, DeviceInfo* info) {
+cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, const double2* __restrict__ partial, int used, int cap,
+                 int n, int s, double theta, uint8_t* flags, uint8_t* flags2, DeviceInfo* info, int with_b) {
     __shared__ double2 e[kMaxN], h[kMaxN], tw[kMaxN];
     __shared__ double2 As[kSmallDim * kSmallDim], Vs[kSmallDim * kSmallDim];
     __shared__ double2 rhs_s[kMaxN / 2], beta_s[kMaxN / 2], coef_s[kMaxN / 2];
@@ -617,10 +731,37 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, int n, int s, 
     const int tid = threadIdx.x;
     const double rsn = 1.0 / sqrt((double)n);
 
-    if (tid < n) {                                         // the projection record: n (re, im) pairs, then n values q_j
-        tw[tid] = cd->twiddle[tid];
-        e[tid] = e_in[tid];
-        qv[tid] = reinterpret_cast<const double*>(e_in + n)[tid];
+    if (tid < n) tw[tid] = cd->twiddle[tid];
+    if (e_in != nullptr) {                                 // the projection record: n (re, im) pairs, then n values q_j
+        if (tid < n) {
+            e[tid] = e_in[tid];
+            qv[tid] = reinterpret_cast<const double*>(e_in + n)[tid];
+        }
+    } else {
+        // the projection's block partials, few enough to add up here: thread (j, part) takes one of the three sums of
+        // node j over the blocks in ascending order, four running sums in rotation (all loads of a round are in flight
+        // together), combined in a fixed order: reproducible
+        const double* __restrict__ qpartial = reinterpret_cast<const double*>(partial + (int64_t)cap * n);
+        for (int idx = tid; idx < 3 * n; idx += blockDim.x) {
+            const int part = idx / n, j = idx - part * n;
+            double acc[4] = {0.0, 0.0, 0.0, 0.0};
+            for (int b0 = 0; b0 < used; b0 += 4) {
+                double v[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int b = (b0 + k < used) ? b0 + k : 0;
+                    const int64_t at = (int64_t)b * n + j;
+                    v[k] = part == 2 ? __ldcg(qpartial + at) : (part == 0 ? __ldcg(&partial[at].x) : __ldcg(&partial[at].y));
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (b0 + k < used) acc[k] += v[k];
+            }
+            const double sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+            if (part == 0) e[j].x = sum;
+            else if (part == 1) e[j].y = sum;
+            else qv[j] = sum;
+        }
     }
     __syncthreads();
     if (tid < n) {
@@ -756,119 +897,11 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, int n, int s, 
         info->locator_margin = margin;
         info->svd_sweeps = sh[3];
     }
-}
-
-// ------------------------------------------------------------------ decode vector
-// With B = [C_L]_{.,V} and A = [C_L]_{.,U}: A A^H = I - B B^H, so the minimum-norm solution of
-// A b_U = e_last is b_U = A^H y, y = e_last + B (I - B^H B)^{-1} B^H e_last, and
-// I - B^H B = [C_R]_{.,V}^H [C_R]_{.,V} is only |V| x |V| (|V| <= 2 s).
-__global__ void __launch_bounds__(kSolveThreads)
-cyc_decode_vector_kernel(CycDevice* cd, const uint8_t* __restrict__ flags, int n, int s, DeviceInfo* info) {
-    __shared__ int vlist[kMaxN], rowbestc[kMaxN], perm_s[kMaxN], sh[4], a_s;
-    __shared__ uint8_t fl[kMaxN];
-    __shared__ double rowbest[kMaxN];
-    __shared__ double2 y[kMaxN], tw[kMaxN], x_s[kMaxN], b_s[kMaxN];
-    __shared__ double2 As[kSmallDim * (kSmallDim + 1)];
-    const int tid = threadIdx.x;
-    const int rows = n - 2 * s, L = rows - 1;
-    const double rsn = 1.0 / sqrt((double)n);
-    if (tid < n) {
-        tw[tid] = cd->twiddle[tid];
-        fl[tid] = flags[tid];
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int a = 0;
-        for (int j = 0; j < n; ++j)
-            if (fl[j]) vlist[a++] = j;
-        a_s = a;
-    }
-    __syncthreads();
-    const int a = a_s;
-    if (a > 2 * s) {                                       // fewer than n - 2 s rows left: no b exists
-        if (tid < n) cd->b[tid] = make_double2(0.0, 0.0);
-        if (tid == 0) {
-            info->n_active = 0; info->n_flagged = a; info->status = DRACO_ETOOMANY;
-            info->im_residual_bits = 0ull; info->re_max_bits = 0ull;
-        }
-        return;
-    }
-    double2* x = x_s;
-    if (a > 0) {
-        const bool small = a <= kSmallDim;
-        double2* A = small ? As : cd->work;
-        for (int idx = tid; idx < a * (a + 1); idx += blockDim.x) {
-            const int p = idx / (a + 1), q = idx % (a + 1);
-            double2 val;
-            if (q < a) {                                   // (1/n) sum_{m >= n-2s} w^(m (v_q - v_p))
-                int dv = vlist[q] - vlist[p];
-                if (dv < 0) dv += n;
-                double re = 0.0, im = 0.0;
-                int k = ((n - 2 * s) * dv) % n;
-                for (int m = n - 2 * s; m < n; ++m) {
-                    const double2 w = tw[k];
-                    re += w.x;
-                    im += w.y;
-                    k += dv;
-                    if (k >= n) k -= n;
-                }
-                val = make_double2(re / n, im / n);
-            } else {                                       // conj(C[L][v_p])
-                const double2 w = tw[(L * vlist[p]) % n];
-                val = make_double2(w.x * rsn, -w.y * rsn);
-            }
-            A[idx] = val;
-        }
+    if (with_b) {                                          // the decode vector for the V just found, same launch
+        __shared__ uint8_t fl_s[kMaxN];
+        if (tid < n) fl_s[tid] = flagged ? 1 : 0;
         __syncthreads();
-        if (small) {
-            if (tid < 32) block_gauss_jordan<true>(A, a, 0.0, x, perm_s, rowbest, rowbestc, sh);
-            __syncthreads();
-        } else {
-            block_gauss_jordan<false>(A, a, 0.0, x, perm_s, rowbest, rowbestc, sh);
-        }
-    }
-    if (tid < rows) {
-        double re = (tid == L) ? 1.0 : 0.0, im = 0.0;
-        for (int p = 0; p < a; ++p) {
-            const double2 w = tw[(tid * vlist[p]) % n];
-            const double2 q = cmul(w, x[p]);
-            re += q.x * rsn;
-            im += q.y * rsn;
-        }
-        y[tid] = make_double2(re, im);
-    }
-    __syncthreads();
-    if (tid < n) {
-        double2 b = make_double2(0.0, 0.0);
-        if (!fl[tid]) {
-            double re = 0.0, im = 0.0;
-            int k = 0;                                     // (m tid) mod n
-            for (int m = 0; m < rows; ++m) {
-                const double2 q = cmulc(y[m], tw[k]);
-                re += q.x;
-                im += q.y;
-                k += tid;
-                if (k >= n) k -= n;
-            }
-            b = make_double2(re * rsn, im * rsn);
-        }
-        cd->b[tid] = b;
-        b_s[tid] = b;
-    }
-    __syncthreads();
-    // the active rows in ascending order: position = number of unflagged nodes before this one
-    if (tid < n && !fl[tid]) {
-        int k = 0;
-        for (int j = 0; j < tid; ++j) k += fl[j] ? 0 : 1;
-        cd->active[k] = tid;
-        cd->b_active[k] = b_s[tid];
-    }
-    if (tid == 0) {
-        info->n_active = n - a;
-        info->n_flagged = a;
-        info->im_residual_bits = 0ull;                     // the recovery kernel's blocks merge their maxima into these
-        info->re_max_bits = 0ull;
-        if (info->status == DRACO_ETOOMANY) info->status = DRACO_OK;
+        decode_vector_body(cd, fl_s, n, s, info);
     }
 }
 
@@ -879,13 +912,20 @@ int project_grid_size(int sm_count, int) { return sm_count * 4; }
 int project_grid_size(int sm_count) { return sm_count * 4; }
 
 // All launches of one projection: n <= 16 the few-rows kernel, n <= 64 one launch of the tile kernel, otherwise two
-// launches of it over half the rows each.  partial: [grid][n] double2 followed by [grid][n] double.
-static cudaError_t launch_project_kernels(int grid, cudaStream_t st, const float2* R, const float* f, int64_t len,
-                                          int64_t ld, int n, double2* partial, int accumulate) {
+// launches of it over half the rows each.  partial: [cap][n] double2 followed by [cap][n] double.  No more blocks
+// are launched than have work (a tile each, or eight 256-coordinate chunks each in the few-rows kernel): short
+// vectors then leave a handful of partials instead of several hundred zeros.  Returns the grid used in *grid_used.
+static cudaError_t launch_project_kernels(int cap, cudaStream_t st, const float2* R, const float* f, int64_t len,
+                                          int64_t ld, int n, double2* partial, int accumulate, int* grid_used) {
     const bool vec2 = (ld % 2 == 0);
+    const int64_t work = n <= 16 ? (len + 256 * kProjectWarps - 1) / (256 * kProjectWarps)
+                                 : (len + kProjectTile - 1) / kProjectTile;
+    int grid = cap;
+    if (work < grid) grid = (int)(work < 1 ? 1 : work);
+    *grid_used = grid;
     if (n <= 16) {
-        if (vec2) cyc_project_fewrows_kernel<true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, partial, accumulate);
-        else cyc_project_fewrows_kernel<false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, partial, accumulate);
+        if (vec2) cyc_project_fewrows_kernel<true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, partial, cap, accumulate);
+        else cyc_project_fewrows_kernel<false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, partial, cap, accumulate);
         return cudaGetLastError();
     }
     const int parts = n <= 64 ? 1 : 2;
@@ -893,11 +933,11 @@ static cudaError_t launch_project_kernels(int grid, cudaStream_t st, const float
     for (int row0 = 0; row0 < n; row0 += per) {
         const int nrows = (n - row0) < per ? (n - row0) : per;
         if (nrows <= 32) {
-            if (vec2) cyc_project_kernel<4, true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, accumulate);
-            else cyc_project_kernel<4, false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, accumulate);
+            if (vec2) cyc_project_kernel<4, true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
+            else cyc_project_kernel<4, false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
         } else {
-            if (vec2) cyc_project_kernel<8, true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, accumulate);
-            else cyc_project_kernel<8, false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, accumulate);
+            if (vec2) cyc_project_kernel<8, true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
+            else cyc_project_kernel<8, false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
         }
         const cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;
@@ -905,28 +945,54 @@ static cudaError_t launch_project_kernels(int grid, cudaStream_t st, const float
     return cudaSuccess;
 }
 
+// accumulate: add to the partials of the plan's earlier launches (column chunks of one vector).  A chunk that needs
+// more blocks than any before it finds the extra slots cleared first.
 int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t len, int64_t ld, bool accumulate,
                        cudaStream_t st) {
-    DRACO_CUDA(launch_project_kernels(p->project_grid, st, R, f, len, ld, p->n, p->partial_dev, accumulate ? 1 : 0));
+    const int cap = p->project_grid;
+    const int64_t work = p->n <= 16 ? (len + 256 * kProjectWarps - 1) / (256 * kProjectWarps)
+                                    : (len + kProjectTile - 1) / kProjectTile;
+    const int want = (int)(work < cap ? (work < 1 ? 1 : work) : cap);
+    if (!accumulate) p->project_used = 0;
+    if (accumulate && want > p->project_used) {
+        const size_t n = (size_t)p->n;
+        DRACO_CUDA(cudaMemsetAsync(p->partial_dev + (size_t)p->project_used * n, 0,
+                                   sizeof(double2) * n * (size_t)(want - p->project_used), st));
+        double* q = reinterpret_cast<double*>(p->partial_dev + (size_t)cap * n);
+        DRACO_CUDA(cudaMemsetAsync(q + (size_t)p->project_used * n, 0, sizeof(double) * n * (size_t)(want - p->project_used), st));
+    }
+    int used = 0;
+    DRACO_CUDA(launch_project_kernels(cap, st, R, f, len, ld, p->n, p->partial_dev, accumulate ? 1 : 0, &used));
+    if (used > p->project_used) p->project_used = used;
     return DRACO_OK;
 }
 
 int launch_cyc_project_finish(draco_plan* p, double2* e_out, cudaStream_t st) {
-    cyc_reduce_partials_kernel<<<p->n, kReduceThreads, 0, st>>>(p->partial_dev, p->project_grid, p->n,
+    cyc_reduce_partials_kernel<<<p->n, kReduceThreads, 0, st>>>(p->partial_dev, p->project_used, p->project_grid, p->n,
                                                                 reinterpret_cast<double*>(e_out));
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }
 
-// e == nullptr: the record of the plan's own projection (launch_cyc_project) is formed first
-int launch_cyc_solve(draco_plan* p, const double2* e, uint8_t* flags, cudaStream_t st) {
+// e == nullptr: the record of the plan's own projection (launch_cyc_project) is formed first: by the locator kernel
+// itself when the projection left few block partials (short vectors, where every launch counts), by the reduction
+// kernel otherwise.  with_b: the decode vector for the set V just found is formed in the same launch.
+int launch_cyc_solve(draco_plan* p, const double2* e, uint8_t* flags, bool with_b, cudaStream_t st) {
+    const double2* partial = nullptr;
+    int used = 0;
     if (!e) {
-        double2* own = reinterpret_cast<double2*>(p->cyc_dev->record);      // address arithmetic only: cyc_dev is a device pointer
-        const int rc = launch_cyc_project_finish(p, own, st);
-        if (rc != DRACO_OK) return rc;
-        e = own;
+        if (p->project_used <= kFusedReduceMax) {
+            partial = p->partial_dev;
+            used = p->project_used;
+        } else {
+            double2* own = reinterpret_cast<double2*>(p->cyc_dev->record);  // address arithmetic only: cyc_dev is a device pointer
+            const int rc = launch_cyc_project_finish(p, own, st);
+            if (rc != DRACO_OK) return rc;
+            e = own;
+        }
     }
-    cyc_solve_kernel<<<1, kSolveThreads, 0, st>>>(p->cyc_dev, e, p->n, p->s, p->theta, flags, p->flags_dev, p->info_dev);
+    cyc_solve_kernel<<<1, kSolveThreads, 0, st>>>(p->cyc_dev, e, partial, used, p->project_grid, p->n, p->s, p->theta, flags,
+                                                  p->flags_dev, p->info_dev, with_b ? 1 : 0);
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }
@@ -990,10 +1056,11 @@ extern "C" int draco_cyc_project_noalloc(int n, int64_t d, const void* R, const 
     if (grid < 1) grid = 1;
     cudaStream_t st = (cudaStream_t)stream;
     const float2* Rc = static_cast<const float2*>(R);
-    // Every block writes its n partials (zeros if it had no tile), so nothing has to be cleared
-    // between calls even though the array keeps the previous call's contents.
-    DRACO_CUDA(launch_project_kernels(grid, st, Rc, f, d, d, n, partial, 0));
-    cyc_reduce_partials_kernel<<<n, kReduceThreads, 0, st>>>(partial, grid, n, e);
+    // Every block that is launched writes its n partials and only those are read back, so nothing has
+    // to be cleared between calls even though the array keeps the previous call's contents.
+    int used = 0;
+    DRACO_CUDA(launch_project_kernels(grid, st, Rc, f, d, d, n, partial, 0, &used));
+    cyc_reduce_partials_kernel<<<n, kReduceThreads, 0, st>>>(partial, used, grid, n, e);
     DRACO_CUDA(cudaGetLastError());
     return DRACO_OK;
 }

@@ -241,7 +241,7 @@ int draco_cyc_project(draco_plan* plan, const void* R, const float* f, double* e
 
 int draco_cyc_locate_from_projection(draco_plan* plan, const double* e, uint8_t* flags, void* stream) {
     if (!plan || !is_cyc(plan) || !e || !flags || !aligned16(e)) return DRACO_EINVAL;
-    return launch_cyc_solve(plan, (const double2*)e, flags, (cudaStream_t)stream);
+    return launch_cyc_solve(plan, (const double2*)e, flags, false, (cudaStream_t)stream);
 }
 
 int draco_locate(draco_plan* plan, const void* R, const float* f, uint8_t* flags, void* stream) {
@@ -252,7 +252,7 @@ int draco_locate(draco_plan* plan, const void* R, const float* f, uint8_t* flags
     if (!f || !aligned16(f)) return DRACO_EINVAL;
     int rc = launch_cyc_project(plan, (const float2*)R, f, vec_len(plan), vec_len(plan), false, st);
     if (rc != DRACO_OK) return rc;
-    return launch_cyc_solve(plan, nullptr, flags, st);
+    return launch_cyc_solve(plan, nullptr, flags, false, st);
 }
 
 int draco_decode(draco_plan* plan, const void* R, const uint8_t* flags, float* u, void* stream) {
@@ -283,9 +283,12 @@ int draco_locate_decode(draco_plan* plan, const void* R, const float* f, uint8_t
     cudaStream_t st = (cudaStream_t)stream;
     if (plan->code == DRACO_REP)
         return launch_rep_vote(plan, (const float*)R, plan->d, plan->d, u, nullptr, flags, true, st);
-    int rc = draco_locate(plan, R, f, flags, stream);
+    // projection, then syndromes / solve / support / decode vector in one launch, then the recovery
+    if (!f || !aligned16(f)) return DRACO_EINVAL;
+    int rc = launch_cyc_project(plan, (const float2*)R, f, vec_len(plan), vec_len(plan), false, st);
+    if (rc == DRACO_OK) rc = launch_cyc_solve(plan, nullptr, flags, true, st);
     if (rc != DRACO_OK) return rc;
-    return draco_decode(plan, R, flags, u, stream);
+    return launch_cyc_recover(plan, (const float2*)R, vec_len(plan), vec_len(plan), u, is_packed(plan) ? plan->d : 0, st);
 }
 
 int draco_cyc_decode_vector(draco_plan* plan, double* b_host, void* stream) {
@@ -420,8 +423,7 @@ int draco_pipeline_host(draco_plan* plan, const float* G_host, const float* f_ho
     }
     int rc;
     if (cyc) {
-        rc = launch_cyc_solve(plan, nullptr, nullptr, st);
-        if (rc == DRACO_OK) rc = launch_cyc_decode_vector(plan, plan->flags_dev, st);
+        rc = launch_cyc_solve(plan, nullptr, nullptr, true, st);
         if (rc == DRACO_OK) rc = launch_cyc_recover(plan, (const float2*)Z, vlen, vlen, plan->u_dev, packed ? d : 0, st);
     } else {
         rc = launch_rep_vote(plan, (const float*)Z, d, d, plan->u_dev, nullptr, nullptr, true, st);

@@ -90,7 +90,8 @@ struct draco_plan {
     draco::CycDevice* cyc_dev;
     draco::DeviceInfo* info_dev;
     double2* partial_dev;             // [project_grid][n]
-    int project_grid;
+    int project_grid;                 // capacity of partial_dev in blocks
+    int project_used;                 // blocks whose partials the plan's last projection (all its chunks) filled
     uint8_t* flags_dev;               // [n] internal flags
     uint32_t* mask_dev;               // repetition: disagreement bits, [n] words
     // host-buffer pipeline (allocated on its first call)
@@ -123,7 +124,7 @@ int launch_cyc_encode(const draco_plan* p, const float* G, float2* Z, int64_t le
 int launch_cyc_project(draco_plan* p, const float2* R, const float* f, int64_t len, int64_t ld, bool accumulate,
                        cudaStream_t st);
 int launch_cyc_project_finish(draco_plan* p, double2* e_out, cudaStream_t st);
-int launch_cyc_solve(draco_plan* p, const double2* e, uint8_t* flags, cudaStream_t st);
+int launch_cyc_solve(draco_plan* p, const double2* e, uint8_t* flags, bool with_b, cudaStream_t st);
 int launch_cyc_decode_vector(draco_plan* p, const uint8_t* flags, cudaStream_t st);
 int launch_cyc_recover(draco_plan* p, const float2* R, int64_t len, int64_t ld, float* u, int64_t d_packed,
                        cudaStream_t st, float* w = nullptr, float scale = 0.0f);
