@@ -274,9 +274,27 @@ def cyc_locate_from_projection(e: np.ndarray, q: np.ndarray, n: int, s: int, the
         cutoff sinks into the rounding noise of complex64 vectors);
       * "t_j != 0" cannot be tested in floating point.  Exactly ``rank`` entries
         of t are non-zero in exact arithmetic, so V = the ``rank`` nodes with the
-        largest |t_j| (V is empty when the rank is 0).
+        largest |t_j| (V is empty when the rank is 0);
+      * the paper's vectors are real numbers; a received vector may hold NaN or
+        infinities.  An honest vector is finite, so a node whose e_j or q_j is not
+        finite is an adversary: it is flagged outright and its e_j, q_j are taken as
+        0, which keeps the arithmetic finite (to the locator the node then looks as
+        if it had sent a vector with f R_j = 0, i.e. the error -f z_j: one of the
+        at most s errors it can locate anyway).
     """
-    e = np.asarray(e, dtype=np.complex128)
+    e = np.asarray(e, dtype=np.complex128).copy()
+    q = np.asarray(q, dtype=np.float64).copy()
+    nonfinite = ~(np.isfinite(e.real) & np.isfinite(e.imag) & np.isfinite(q))
+    e[nonfinite] = 0.0
+    q[nonfinite] = 0.0
+    out = _cyc_locate_finite(e, q, n, s, theta)
+    out["flags"] = out["flags"] | nonfinite
+    out["nonfinite"] = nonfinite
+    return out
+
+
+def _cyc_locate_finite(e: np.ndarray, q: np.ndarray, n: int, s: int, theta: float) -> dict:
+    """The steps of phi on a finite projection record (see cyc_locate_from_projection)."""
     C = idft_matrix(n)
     scale = float(np.median(np.sqrt(np.asarray(q, dtype=np.float64))))
     tol = theta * scale

@@ -284,3 +284,37 @@ def test_rank_cutoff_is_measured_against_the_size_of_the_vectors_not_of_their_pr
     R[adv] *= -100
     loc = orc.cyc_locate(R, di.projection_vector(33, d), n, s)
     assert sorted(np.flatnonzero(loc["flags"])) == adv
+
+
+@pytest.mark.parametrize("n,s", [(5, 1), (7, 2), (9, 2)])
+def test_adversaries_sending_nan_or_infinities_are_flagged_and_the_sum_is_exact(n, s):
+    """Definition 2 with "arbitrary" taken at its word: vectors holding NaN or infinities, alone or beside an
+    ordinary reversed-gradient adversary, at every placement of up to s adversaries."""
+    import warnings
+    d = 12
+    G = di.gradient_rows(3, n, d)
+    Z = orc.cyc_encode(G, n, s)
+    f = di.projection_vector(4, d)
+    exact = G.astype(np.float64).sum(axis=0)
+    with warnings.catch_warnings():
+        warnings.simplefilter("ignore")                         # numpy warns about inf - inf on the way
+        for a in range(1, s + 1):
+            for placement in itertools.combinations(range(n), a):
+                for kind in range(3):
+                    R = Z.copy()
+                    for k, j in enumerate(placement):
+                        if kind == 0:
+                            R[j, 3] = np.nan                     # a single NaN entry
+                        elif kind == 1 and k % 2 == 0:
+                            R[j] = np.inf * (1 + 1j)
+                        elif kind == 1:
+                            R[j] = -100 * R[j]                   # an ordinary adversary beside the infinite one
+                        else:
+                            R[j, ::2] = -np.inf
+                            R[j, 1] = np.nan
+                    out = orc.cyc_decode_full(R, f, n, s)
+                    assert set(np.flatnonzero(out["flags"])) == set(placement)
+                    assert np.all(np.isfinite(out["u"]))
+                    assert np.abs(out["u"] - exact).max() <= 1e-4 * np.abs(exact).max()
+    # a clean matrix reports no such node
+    assert not orc.cyc_locate(Z, f, n, s)["nonfinite"].any()
