@@ -138,7 +138,8 @@ int draco_encode(const draco_plan* plan, const float* G, void* Z, void* stream);
  *   cyclic:     V = phi(R): e = f R (fp64 accumulation), the 2 s syndromes e C_R^dagger,
  *               the s x s Toeplitz system for beta (pseudo-inverse solution from an SVD),
  *               the recurrence h_l = sum_u beta_u h_{l+u-s}, t = IDFT(h), V = supp(t)
- *               read as the rank-many largest |t_j|.
+ *               read as the rank-many largest |t_j|.  A node whose vector holds NaN or infinities (its
+ *               projection is then not finite) is flagged outright and counted as having sent f R_j = 0.
  * R: device [n][d].  f: device [d] fp32, the caller's draw of N(1_d, I_d) (cyclic only).
  * flags: device [n] bytes.
  */

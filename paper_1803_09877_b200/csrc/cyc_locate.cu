@@ -764,7 +764,17 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, const double2*
         }
     }
     __syncthreads();
+    // A node whose record is not finite sent NaN or infinities: no honest vector does.  It is flagged outright and
+    // its record taken as zero, which keeps the arithmetic below finite (the node then looks to the locator as if it
+    // had sent a vector with f R_j = 0: one of the at most s errors it locates anyway).
+    __shared__ uint8_t nonfinite[kMaxN];
     if (tid < n) {
+        const bool bad = !(isfinite(e[tid].x) && isfinite(e[tid].y) && isfinite(qv[tid]));
+        nonfinite[tid] = bad ? 1 : 0;
+        if (bad) {
+            e[tid] = make_double2(0.0, 0.0);
+            qv[tid] = 0.0;
+        }
         cd->e[tid] = e[tid];
         mag[tid] = sqrt(qv[tid]);
         h[tid] = make_double2(0.0, 0.0);
@@ -878,6 +888,7 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, const double2*
     }
     if (tid < n) {
         cd->h[tid] = h[tid];
+        flagged = flagged || nonfinite[tid];
         if (flags) flags[tid] = flagged ? 1 : 0;
         if (flags2) flags2[tid] = flagged ? 1 : 0;
         if (flagged) atomicAdd(&count, 1);

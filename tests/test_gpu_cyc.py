@@ -561,3 +561,33 @@ def test_decode_with_null_flags_uses_the_plans_last_locate():
     plan.decode_update(Rd, None, wb, 0.01)
     torch.cuda.synchronize()
     assert torch.equal(wa, wb)
+
+
+@pytest.mark.parametrize("n,s,d", [(15, 2, 6150), (45, 5, 4099)])
+def test_adversaries_sending_nan_or_infinities(n, s, d):
+    """A vector with NaN or infinite entries is flagged outright (its projection is not finite), the others are
+    located as usual, and the sum comes out finite and exact; flags and sum against the oracle on the same R."""
+    dr, plan = _plan(n, s, d)
+    G = di.gradient_rows(31 * n + s, n, d)
+    R = orc.cyc_encode(G, n, s)
+    adv = di.choose_adversaries(5 * n + s, n, s)
+    R[adv[0], 7] = np.nan                                      # one NaN entry in an otherwise honest vector
+    if s > 1:
+        R[adv[1], ::3] = np.inf * (1 - 1j)
+    for j in adv[2:]:
+        R[j] = -100 * R[j]
+    f = di.projection_vector(77, d)
+    import warnings
+    with warnings.catch_warnings():
+        warnings.simplefilter("ignore")
+        want = orc.cyc_decode_full(R, f, n, s)
+    assert sorted(np.flatnonzero(want["flags"])) == adv.tolist() and want["nonfinite"].sum() == min(s, 2)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan.locate_decode(dev(R), dev(f), flags, u)
+    info = plan.info()
+    np.testing.assert_array_equal(host(flags).astype(bool), want["flags"])
+    assert info["status"] == 0 and info["n_flagged"] == s and info["locator_rank"] == want["rank"]
+    assert np.all(np.isfinite(host(u)))
+    assert normwise(host(u), want["u"]) <= 1e-6
+    assert normwise(host(u), G.astype(np.float64).sum(axis=0)) <= (1e-4 if n <= 15 else 1e-2)
