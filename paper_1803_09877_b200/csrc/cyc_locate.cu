@@ -81,6 +81,15 @@ cyc_project_kernel(const float2* __restrict__ R, const float* __restrict__ f, in
     __shared__ double2 es[kProjectWarps * RPW];
     __shared__ double qs[kProjectWarps * RPW];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Short vectors have fewer tiles than the device has SMs; the launch then splits the rows over gridDim.y as well
+    // (whole multiples of the 8 warps' rows), every (tile, node) partial still being written by exactly one block.
+    if (gridDim.y > 1) {
+        const int per = (((nrows + (int)gridDim.y - 1) / (int)gridDim.y + kProjectWarps - 1) / kProjectWarps) * kProjectWarps;
+        const int skip = (int)blockIdx.y * per;
+        if (skip >= nrows) return;
+        row0 += skip;
+        nrows = (nrows - skip) < per ? (nrows - skip) : per;
+    }
     if (lane == 0) {
 #pragma unroll
         for (int r = 0; r < RPW; ++r) {
@@ -445,7 +454,12 @@ __device__ int block_jacobi_pinv(double2* A, double2* V, const double2* rhs, int
             if (tid < sp / 2) {
                 int a, b;
                 if (tid == 0) { a = sp - 1; b = step; }
-                else { a = (step + tid) % (sp - 1); b = (step - tid + (sp - 1)) % (sp - 1); }
+                else {                                    // (step +- tid) mod (sp - 1); both step and tid are below sp - 1
+                    a = step + tid;
+                    if (a >= sp - 1) a -= sp - 1;
+                    b = step - tid;
+                    if (b < 0) b += sp - 1;
+                }
                 const int p = a < b ? a : b, q = a < b ? b : a;
                 double2* ap = A + p * sp;
                 double2* aq = A + q * sp;
@@ -531,7 +545,12 @@ __device__ int warp_jacobi_pinv(double2* A, double2* V, const double2* rhs, int 
             if (act) {
                 int a, b;
                 if (pair == 0) { a = sp - 1; b = step; }
-                else { a = (step + pair) % (sp - 1); b = (step - pair + (sp - 1)) % (sp - 1); }
+                else {                                    // (step +- pair) mod (sp - 1); both are below sp - 1
+                    a = step + pair;
+                    if (a >= sp - 1) a -= sp - 1;
+                    b = step - pair;
+                    if (b < 0) b += sp - 1;
+                }
                 p = a < b ? a : b;
                 q = a < b ? b : a;
             }
@@ -941,14 +960,23 @@ static cudaError_t launch_project_kernels(int cap, cudaStream_t st, const float2
     }
     const int parts = n <= 64 ? 1 : 2;
     const int per = (n + parts - 1) / parts;
+    // fewer tiles than an eighth of the blocks the device takes: spread the rows over gridDim.y too (latency of short vectors)
+    int ysplit = 1;
+    if (grid * 8 <= cap) {
+        ysplit = (per + kProjectWarps - 1) / kProjectWarps;
+        const int room = cap / (2 * grid);
+        if (ysplit > room) ysplit = room;
+        if (ysplit < 1) ysplit = 1;
+    }
+    const dim3 grid2(grid, ysplit);
     for (int row0 = 0; row0 < n; row0 += per) {
         const int nrows = (n - row0) < per ? (n - row0) : per;
         if (nrows <= 32) {
-            if (vec2) cyc_project_kernel<4, true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
-            else cyc_project_kernel<4, false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
+            if (vec2) cyc_project_kernel<4, true><<<grid2, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
+            else cyc_project_kernel<4, false><<<grid2, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
         } else {
-            if (vec2) cyc_project_kernel<8, true><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
-            else cyc_project_kernel<8, false><<<grid, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
+            if (vec2) cyc_project_kernel<8, true><<<grid2, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
+            else cyc_project_kernel<8, false><<<grid2, kThreads, 0, st>>>(R, f, len, ld, n, row0, nrows, partial, cap, accumulate);
         }
         const cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;

@@ -104,10 +104,13 @@ int grid_for(int64_t work, int sm_count, int per_sm) {
     return (int)want;
 }
 
-int device_sm_count() {
+int device_sm_count() {                     // of the current device; looked up once per device
+    static int cached[64] = {};
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 1;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 1;
+    if (dev >= 0 && dev < 64 && cached[dev] > 0) return cached[dev];
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return 1;
+    if (dev >= 0 && dev < 64) cached[dev] = sms;
     return sms;
 }
 
