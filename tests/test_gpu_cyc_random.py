@@ -1,7 +1,9 @@
 """Cyclic code on many small random cases: shapes, adversary counts, attack models and seeds drawn from one seeded
-stream.  The GPU's flags must equal the oracle's on the very same received matrix in every case that does not sit on
-the rank cutoff, and where both find the planted adversaries the decoded sum must sit on the oracle's own complex64
-floor."""
+stream.  The GPU's flags and rank must equal the oracle's on the very same received matrix in **every** case, those
+included where a singular value sits at the rank cutoff or the flagged and unflagged |t_j| are alike: the device forms
+the projection exactly (fp32 x fp32 products in fp64), so both sides see the same rounding noise and decide alike.
+Where both find the planted adversaries the decoded sum must sit on the oracle's own complex64 floor, and a set that is
+not the planted one never comes back with a clean status."""
 import numpy as np
 import pytest
 import torch
@@ -13,7 +15,7 @@ from gpu_util import dev, host, normwise
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("stream_seed", [11, 12])
+@pytest.mark.parametrize("stream_seed", [11, 12, 13])
 def test_random_small_cases_match_the_oracle(stream_seed):
     import paper_1803_09877_b200 as dr
     rng = np.random.default_rng(stream_seed)
@@ -47,9 +49,7 @@ def test_random_small_cases_match_the_oracle(stream_seed):
             warned += 1
             assert info["status"] in (dr.binding.EUNSURE, dr.binding.ETOOMANY), what
         if any(tol / 3 < x < 3 * tol for x in want.get("sv", [])) or (0 < want["rank"] < n and want["margin"] < 10):
-            on_the_edge += 1         # a singular value at the rank cutoff, or |t| of flagged and unflagged nodes alike:
-            plan.close()             # rounding decides, and the two sides round differently
-            continue
+            on_the_edge += 1         # a singular value at the rank cutoff, or |t| of flagged and unflagged nodes alike: counted
         np.testing.assert_array_equal(host(flags).astype(bool), want["flags"], err_msg=what)
         assert info["locator_rank"] == want["rank"], what
         if sorted(np.flatnonzero(want["flags"]).tolist()) == adv:
@@ -59,8 +59,8 @@ def test_random_small_cases_match_the_oracle(stream_seed):
             assert normwise(host(u), exact) <= 2.0 * floor + 1e-6, what
             assert info["im_residual"] <= 0.05 * info["re_max"], what
         plan.close()
-    # the rest: clustered adversaries beyond what complex64 vectors can carry
-    assert on_the_edge <= 4 and both_found >= 54
+    # the rest: clustered adversaries beyond what complex64 vectors can carry (measured: 59 or 60 of 60 found)
+    assert on_the_edge <= 6 and both_found >= 56
     assert warned <= 60 - both_found
 
 
@@ -97,8 +97,6 @@ def test_random_small_packed_cases_match_the_oracle():
         tol = 1e-6 * want["scale"]
         if any(tol / 3 < x < 3 * tol for x in want.get("sv", [])) or (0 < want["rank"] < n and want["margin"] < 10):
             on_the_edge += 1
-            plan.close()
-            continue
         np.testing.assert_array_equal(host(flags).astype(bool), want["flags"], err_msg=what)
         assert info["locator_rank"] == want["rank"], what
         if sorted(np.flatnonzero(want["flags"]).tolist()) == adv:
@@ -108,4 +106,4 @@ def test_random_small_packed_cases_match_the_oracle():
             exact = G.astype(np.float64).sum(axis=0)
             assert normwise(host(u), exact) <= 2.0 * normwise(uo, exact) + 1e-6, what
         plan.close()
-    assert on_the_edge <= 4 and both_found >= 54
+    assert on_the_edge <= 6 and both_found >= 56
