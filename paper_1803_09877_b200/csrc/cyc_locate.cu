@@ -54,11 +54,6 @@ __device__ __forceinline__ double warp_sum(double a) {
     for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
     return a;
 }
-__device__ __forceinline__ float warp_sum(float a) {
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
-    return a;
-}
 // Block partials: [cap][n] double2 (e) followed by [cap][n] double (q); cap = the capacity of the buffer in blocks,
 // of which a launch fills the first gridDim.x.
 __device__ __forceinline__ double* q_partials(double2* partial, int cap, int n) {

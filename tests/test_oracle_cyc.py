@@ -318,3 +318,26 @@ def test_adversaries_sending_nan_or_infinities_are_flagged_and_the_sum_is_exact(
                     assert np.abs(out["u"] - exact).max() <= 1e-4 * np.abs(exact).max()
     # a clean matrix reports no such node
     assert not orc.cyc_locate(Z, f, n, s)["nonfinite"].any()
+
+
+def test_projection_and_energy_closed_forms():
+    """e = f R and q_j = sum_i |R[j][i]|^2 on inputs whose sums are known in closed form: rows of unit-modulus
+    geometric sequences R[j][i] = exp(2 pi i j i / m) scaled by a_j, with f = 1 and with f = the ramp 0, 1, 2, ..."""
+    n, d, m = 6, 40, 8
+    a = np.array([1.0, 2.0, 0.5, 3.0, 1.5, 0.25])
+    i = np.arange(d)
+    z = np.exp(2j * np.pi * np.arange(n) / m)                       # ratio of row j's geometric sequence
+    R = a[:, None] * z[:, None] ** i[None, :]
+    # q: every entry of row j has modulus a_j
+    np.testing.assert_allclose(orc.cyc_project_energy(R), d * a ** 2, rtol=1e-13)
+    # f = 1: geometric sum (row 0 has ratio 1); d = 40 is a multiple of m / gcd(j, m) for every j, so the others vanish
+    e1 = orc.cyc_project(R, np.ones(d))
+    want1 = np.where(np.arange(n) == 0, a * d, 0.0)
+    np.testing.assert_allclose(e1, want1, atol=1e-12)
+    # f = ramp: sum_i i z^i = z (1 - d z^(d-1) + (d-1) z^d) / (1 - z)^2 for z != 1, d (d - 1) / 2 for z = 1
+    e2 = orc.cyc_project(R, i.astype(np.float64))
+    zz = z[1:]
+    want2 = np.concatenate([[a[0] * d * (d - 1) / 2], a[1:] * zz * (1 - d * zz ** (d - 1) + (d - 1) * zz ** d) / (1 - zz) ** 2])
+    np.testing.assert_allclose(e2, want2, rtol=1e-11, atol=1e-11)
+    # a transposed or conjugated operand would not pass: the ramp sum of row 1 has a non-zero imaginary part of known sign
+    assert want2[1].imag < -1.0 and abs(e2[1].imag - want2[1].imag) < 1e-9
