@@ -591,3 +591,39 @@ def test_adversaries_sending_nan_or_infinities(n, s, d):
     assert np.all(np.isfinite(host(u)))
     assert normwise(host(u), want["u"]) <= 1e-6
     assert normwise(host(u), G.astype(np.float64).sum(axis=0)) <= (1e-4 if n <= 15 else 1e-2)
+
+
+def test_host_pipeline_over_several_column_chunks():
+    """d large enough that draco_pipeline_host streams G in three column chunks (the last one ragged): the projection
+    then accumulates over the chunks' launches.  Same worker vectors, flags and sum as the device-resident path."""
+    import paper_1803_09877_b200 as dr
+    n, s, d = 45, 3, 3_100_004
+    plan = dr.Plan(n, s, d, dr.CYC)
+    seed = 777
+    G = torch.empty((n, d), dtype=torch.float32, device="cuda")
+    dr.generate(G, n, d, seed=seed)
+    f = torch.empty(d, dtype=torch.float32, device="cuda")
+    dr.generate(f, 1, d, mean=1.0, std=1.0, seed=seed + 3)
+    adv = di.choose_adversaries(seed + 1, n, s)
+    Gh, fh = G.cpu().numpy(), f.cpu().numpy()
+    Z = torch.empty((n, 2 * d), dtype=torch.float32, device="cuda")
+    u_host = np.empty(d, dtype=np.float32)
+    flags_host = np.empty(n, dtype=np.uint8)
+    info = plan.pipeline_host(Gh.ctypes.data, fh.ctypes.data, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed + 2, Z,
+                              u_host.ctypes.data, flags_host.ctypes.data)
+    assert info["status"] == 0 and sorted(np.flatnonzero(flags_host)) == adv.tolist() and info["locator_rank"] == s
+    Z2 = torch.empty_like(Z)
+    plan2 = dr.Plan(n, s, d, dr.CYC)
+    plan2.encode(G, Z2)
+    plan2.corrupt(Z2, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=seed + 2)
+    flags = torch.empty(n, dtype=torch.uint8, device="cuda")
+    u = torch.empty(d, dtype=torch.float32, device="cuda")
+    plan2.locate_decode(Z2, f, flags, u)
+    torch.cuda.synchronize()
+    assert torch.equal(Z, Z2)
+    np.testing.assert_array_equal(host(flags), flags_host)
+    np.testing.assert_array_equal(host(u), u_host)             # same flags, same decode vector, same rows: same bits
+    # and the sum itself on a sample, against the exact one
+    idx = np.unique(np.concatenate([np.arange(64), np.arange(d - 64, d), np.random.default_rng(1).integers(0, d, 5000)]))
+    exact = Gh[:, idx].astype(np.float64).sum(axis=0)
+    assert normwise(u_host[idx], exact) <= 2e-3                # complex64 floor at (45, 3) is about 2e-4
