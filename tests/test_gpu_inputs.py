@@ -44,3 +44,23 @@ def test_corrupt_matches_numpy(code):
     want = di.apply_adversaries(R0.copy(), adv, model, param, seed=99)
     got = host(Rd, complex64=(code == dr.CYC))
     np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_corruptor_rejects_duplicate_and_out_of_range_nodes():
+    """All adversarial rows are rewritten by one launch, so a node may appear once only."""
+    import paper_1803_09877_b200 as dr
+    from paper_1803_09877_b200 import binding
+    n, s, d = 9, 2, 64
+    plan = dr.Plan(n, s, d, dr.REP)
+    Z = torch.zeros((n, d), dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.DracoError, match="invalid argument"):
+        plan.corrupt(Z, [3, 3], [dr.ADV_CONST] * 2, [1.0] * 2)
+    with pytest.raises(binding.DracoError, match="invalid argument"):
+        plan.corrupt(Z, [9], [dr.ADV_CONST], [1.0])
+    with pytest.raises(binding.DracoError, match="invalid argument"):
+        plan.corrupt(Z, [1], [7], [1.0])
+    torch.cuda.synchronize()
+    assert float(Z.abs().max()) == 0.0                     # nothing was launched
+    plan.corrupt(Z, [1, 8], [dr.ADV_CONST] * 2, [2.0, 3.0])
+    torch.cuda.synchronize()
+    assert Z[1].eq(2.0).all() and Z[8].eq(3.0).all() and float(Z[[0, 2, 3, 4, 5, 6, 7]].abs().max()) == 0.0
