@@ -63,7 +63,9 @@ __device__ __forceinline__ void update_vals(float* ptr, const float (&x)[2], flo
 __device__ __forceinline__ void update_vals(float* ptr, const float (&x)[1], float scale) { ptr[0] = fmaf(-scale, x[0], ptr[0]); }
 
 // ---------------------------------------------------------------- encode
-template <int MMAX, int VEC>
+// MMAX > 0: groups of at most MMAX members, GB groups fetched together so that about 16 rows are in flight per
+// thread whatever the group size (as in the vote kernel); MMAX == 0: larger groups, members streamed.
+template <int MMAX, int VEC, int GB>
 __global__ void __launch_bounds__(kThreads)
 rep_encode_kernel(const float* __restrict__ G, float* __restrict__ Z, int64_t len, int64_t ldg, int64_t ldz,
                   GroupTable gt) {
@@ -71,23 +73,37 @@ rep_encode_kernel(const float* __restrict__ G, float* __restrict__ Z, int64_t le
     const int64_t stride = (int64_t)gridDim.x * kThreads;
     for (int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x; v < nvec; v += stride) {
         const int64_t col = v * VEC;
-        for (int g = 0; g < gt.num_groups; ++g) {
-            const int first = gt.first[g], m = gt.size[g];
-            float acc[VEC];
-            if constexpr (MMAX > 0) {
-                Pack<VEC> val[MMAX > 0 ? MMAX : 1];
+        if constexpr (MMAX > 0) {
+            for (int g0 = 0; g0 < gt.num_groups; g0 += GB) {
+                Pack<VEC> val[GB][MMAX];
 #pragma unroll
-                for (int k = 0; k < MMAX; ++k)
-                    if (k < m) load_pack(val[k], reinterpret_cast<const uint32_t*>(G + (int64_t)(first + k) * ldg + col));
+                for (int b = 0; b < GB; ++b)
+                    if (g0 + b < gt.num_groups) {
+                        const int first = gt.first[g0 + b], m = gt.size[g0 + b];
 #pragma unroll
-                for (int c = 0; c < VEC; ++c) acc[c] = __uint_as_float(val[0].get(c));
-#pragma unroll
-                for (int k = 1; k < MMAX; ++k)
-                    if (k < m) {
-#pragma unroll
-                        for (int c = 0; c < VEC; ++c) acc[c] = __fadd_rn(acc[c], __uint_as_float(val[k].get(c)));
+                        for (int k = 0; k < MMAX; ++k)
+                            if (k < m) load_pack(val[b][k], reinterpret_cast<const uint32_t*>(G + (int64_t)(first + k) * ldg + col));
                     }
-            } else {
+#pragma unroll
+                for (int b = 0; b < GB; ++b)
+                    if (g0 + b < gt.num_groups) {
+                        const int first = gt.first[g0 + b], m = gt.size[g0 + b];
+                        float acc[VEC];
+#pragma unroll
+                        for (int c = 0; c < VEC; ++c) acc[c] = __uint_as_float(val[b][0].get(c));
+#pragma unroll
+                        for (int k = 1; k < MMAX; ++k)
+                            if (k < m) {
+#pragma unroll
+                                for (int c = 0; c < VEC; ++c) acc[c] = __fadd_rn(acc[c], __uint_as_float(val[b][k].get(c)));
+                            }
+                        for (int k = 0; k < m; ++k) store_vals(Z + (int64_t)(first + k) * ldz + col, acc);
+                    }
+            }
+        } else {
+            for (int g = 0; g < gt.num_groups; ++g) {
+                const int first = gt.first[g], m = gt.size[g];
+                float acc[VEC];
                 Pack<VEC> x;
                 load_pack(x, reinterpret_cast<const uint32_t*>(G + (int64_t)first * ldg + col));
 #pragma unroll
@@ -97,8 +113,8 @@ rep_encode_kernel(const float* __restrict__ G, float* __restrict__ Z, int64_t le
 #pragma unroll
                     for (int c = 0; c < VEC; ++c) acc[c] = __fadd_rn(acc[c], __uint_as_float(x.get(c)));
                 }
+                for (int k = 0; k < m; ++k) store_vals(Z + (int64_t)(first + k) * ldz + col, acc);
             }
-            for (int k = 0; k < m; ++k) store_vals(Z + (int64_t)(first + k) * ldz + col, acc);
         }
     }
 }
@@ -334,15 +350,18 @@ int launch_rep_encode(const draco_plan* p, const float* G, float* Z, int64_t len
     const bool vec4 = (len % 4 == 0) && (ldg % 4 == 0) && (ldz % 4 == 0);
     const int64_t nvec = vec4 ? len / 4 : len;
     const int grid = grid_for(nvec, p->sm_count, 8);
-#define DRACO_ENC(MM, VV) rep_encode_kernel<MM, VV><<<grid, kThreads, 0, st>>>(G, Z, len, ldg, ldz, gt)
+#define DRACO_ENC(MM, VV, GG) rep_encode_kernel<MM, VV, GG><<<grid, kThreads, 0, st>>>(G, Z, len, ldg, ldz, gt)
     if (vec4) {
-        if (gt.max_size <= 8) DRACO_ENC(8, 4);
-        else if (gt.max_size <= 16) DRACO_ENC(16, 4);
-        else DRACO_ENC(0, 4);
+        if (gt.max_size <= 3) DRACO_ENC(3, 4, 5);
+        else if (gt.max_size <= 4) DRACO_ENC(4, 4, 4);
+        else if (gt.max_size <= 5) DRACO_ENC(5, 4, 2);
+        else if (gt.max_size <= 8) DRACO_ENC(8, 4, 2);
+        else if (gt.max_size <= 16) DRACO_ENC(16, 4, 1);
+        else DRACO_ENC(0, 4, 1);
     } else {
-        if (gt.max_size <= 8) DRACO_ENC(8, 1);
-        else if (gt.max_size <= 16) DRACO_ENC(16, 1);
-        else DRACO_ENC(0, 1);
+        if (gt.max_size <= 8) DRACO_ENC(8, 1, 2);
+        else if (gt.max_size <= 16) DRACO_ENC(16, 1, 1);
+        else DRACO_ENC(0, 1, 1);
     }
 #undef DRACO_ENC
     DRACO_CUDA(cudaGetLastError());
@@ -361,7 +380,9 @@ int launch_rep_vote(draco_plan* p, const float* R, int64_t len, int64_t ld, floa
     rep_vote_kernel<MM, VV, GG, TT><<<grid_for(len / VV, p->sm_count, 8) * (kThreads / TT), TT, 0, st>>>(Rb, len, ld, gt, u, \
                                                                                                         maj, scratch, w, scale)
     if (vec4) {
-        if (gt.max_size <= 4) DRACO_VOTE(4, 4, 4, 256);
+        if (gt.max_size <= 3) DRACO_VOTE(3, 4, 5, 256);             // s = 1: five groups of three = 15 rows in flight
+        else if (gt.max_size <= 4) DRACO_VOTE(4, 4, 4, 256);
+        else if (gt.max_size <= 5) DRACO_VOTE(5, 4, 3, 256);        // s = 2: three groups of five
         else if (gt.max_size <= 8) DRACO_VOTE(8, 4, 2, 256);
         else if (gt.max_size <= 16) DRACO_VOTE(16, 4, 1, 128);      // 16 x 128-bit loads per thread: small blocks keep 3 per SM
         else DRACO_VOTE(0, 4, 1, 256);
