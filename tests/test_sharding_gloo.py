@@ -70,7 +70,7 @@ def test_sharded_locate_and_decode(world, d):
     with socket.socket() as sock:
         sock.bind(("127.0.0.1", 0))
         port = sock.getsockname()[1]
-    manager = mp.Manager()
+    manager = mp.get_context("spawn").Manager()
     result = manager.dict()
     mp.spawn(_worker, args=(world, port, n, s, d, adv, result), nprocs=world, join=True)
     # single-process answer
