@@ -436,7 +436,7 @@ def measure_workload(args, workload, world, rank, with_graph, with_e2e):
 
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per gradient coordinate of the dominant kernel (profiles/)
-DOMINANT_TRAFFIC_PER_COORD = {("cyc", 45, 5): 525.1, ("cycp", 45, 5): 353.6, ("rep", 45, 3): 183.0}
+DOMINANT_TRAFFIC_PER_COORD = {("cyc", 45, 5): 525.1, ("cycp", 45, 5): 353.9, ("rep", 45, 3): 183.0}
 SECONDARY_WORKLOADS = ["rep_n45_s3_d11.7M", "cycp_n45_s5_d60.2M"]
 
 

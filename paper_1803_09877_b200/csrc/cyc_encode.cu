@@ -54,8 +54,10 @@ struct StreamCfg {
 
 // ---------------------------------------------------------------- asynchronous-copy and shared-memory wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async8(uint32_t dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+// The same copy with its source switched off by a predicate (ignore-src: zeros are written, src is not read), so that
+// a lane outside the vector needs no branch around its copies.
+__device__ __forceinline__ void cp_async8_if(uint32_t dst, const void* src, bool on) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, %2, 0;\n\tcp.async.ca.shared.global [%0], [%1], 8, p;\n\t}" ::"r"(dst), "l"(src), "r"((uint32_t)on) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -86,6 +88,7 @@ struct Fetcher {
     const float* G;
     const float* ga;            // this lane's first pair in the next row to fetch
     int64_t boff;               // from there to its second pair: 64, or `half` when PACKED
+    int64_t boff_now;           // the same, 0 while the second pair is switched off
     int64_t strip, nstrips, strip_step, len, ldg;
     int row, n, lane;
     bool act0, act1;            // the pairs lie inside the vector (and the strip exists)
@@ -94,14 +97,17 @@ struct Fetcher {
         const int64_t c = strip * kStrip + 2 * lane;
         act0 = strip < nstrips && c < len;
         act1 = PACKED ? act0 : (strip < nstrips && c + 64 < len);
-        ga = G + c;
+        // switched-off copies still carry an address: keep it inside the matrix (this lane's first pair of strip 0, and
+        // the first pair again for a second pair beyond the row's end)
+        ga = G + (act0 ? c : (int64_t)(2 * lane < len ? 2 * lane : 0));
+        boff_now = act1 ? boff : 0;
         row = 0;
     }
-    // copy this lane's 16 bytes of the next row to shared address dst and close the group (an empty group
-    // when the lane has nothing to copy, so that every thread counts the same groups)
+    // copy this lane's 16 bytes of the next row to shared address dst and close the group (copies of a lane
+    // outside the vector are switched off; every thread counts the same groups)
     __device__ __forceinline__ void fetch(uint32_t dst) {
-        if (act0) cp_async8(dst, ga);
-        if (act1) cp_async8(dst + 8, ga + boff);
+        cp_async8_if(dst, ga, act0);
+        cp_async8_if(dst + 8, ga + boff_now, act1);
         cp_async_commit();
         ga += ldg;
         if (++row == n) {
