@@ -460,7 +460,11 @@ def run_gpu(args):
     ranks = None
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-        mine = {"rank": rank, "device": local, "uuid": str(torch.cuda.get_device_properties(local).uuid)}
+        try:
+            uuid = str(torch.cuda.get_device_properties(local).uuid)
+        except Exception:                       # older runtimes have no uuid field: fall back to the device ordinal
+            uuid = f"ordinal-{local}"
+        mine = {"rank": rank, "device": local, "uuid": uuid}
         gathered = [None] * world
         dist.all_gather_object(gathered, mine)
         ranks = gathered
