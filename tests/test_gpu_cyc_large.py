@@ -184,3 +184,42 @@ def test_decode_vector_with_more_than_16_flags(n, s, d, n_flags):
         flags[free[0]] = 1
         plan.decode(dev(R), dev(flags), u)
         assert plan.info()["status"] == dr.binding.ETOOMANY and float(u.abs().max()) == 0.0
+
+
+# the smallest and the largest shapes the plan accepts: one node, one coordinate, s = (n - 1) / 2 at n = 3 and n = 127 / 128
+@pytest.mark.parametrize("n,s,d", [(1, 0, 1), (1, 0, 7), (2, 0, 3), (3, 1, 1), (3, 1, 2), (127, 63, 5), (128, 63, 9)])
+@pytest.mark.parametrize("code_name", ["CYC", "CYC_PACKED", "REP"])
+def test_degenerate_shapes(n, s, d, code_name):
+    import paper_1803_09877_b200 as dr
+    plan = dr.Plan(n, s, d, getattr(dr, code_name))
+    G = di.gradient_rows(11 * n + d, n, d)
+    exact = G.astype(np.float64).sum(axis=0)
+    flags = torch.full((n,), 9, dtype=torch.uint8, device="cuda")
+    u = torch.full((d,), float("nan"), dtype=torch.float32, device="cuda")
+    if code_name == "REP":
+        Z = torch.empty((n, d), dtype=torch.float32, device="cuda")
+        plan.encode(dev(G), Z)
+        torch.cuda.synchronize()
+        Zo = orc.rep_encode(G, n, s)                         # fp64 sums rounded once; the device adds in fp32, ascending
+        assert np.abs(host(Z) - Zo).max() <= 1e-6 * max(np.abs(Zo).max(), 1e-30)
+        for first, size in orc.rep_groups(n, s):
+            assert (host(Z)[first:first + size].view(np.uint32) == host(Z)[first].view(np.uint32)).all()
+        plan.locate_decode(Z, None, flags, u)
+        info = plan.info()
+        assert not host(flags).any() and info["status"] == 0 and info["no_majority"] == 0
+        assert np.abs(host(u) - exact).max() <= 1e-5 * max(np.abs(exact).max(), 1e-30)
+        return
+    packed = code_name == "CYC_PACKED"
+    h = (d + 1) // 2 if packed else d
+    Z = torch.empty((n, 2 * h), dtype=torch.float32, device="cuda")
+    plan.encode(dev(G), Z)
+    torch.cuda.synchronize()
+    Zo = orc.cyc_encode_packed(G, n, s, dtype=np.complex128) if packed else orc.cyc_encode(G, n, s, dtype=np.complex128)
+    Zg = host(Z, complex64=True)
+    for j in range(n):
+        assert np.abs(Zg[j] - Zo[j]).max() <= 1e-6 * max(np.abs(Zo[j]).max(), 1e-30)
+    f = di.projection_vector(5, h)
+    plan.locate_decode(Z, dev(f), flags, u)
+    info = plan.info()
+    assert not host(flags).any() and info["locator_rank"] == 0 and info["status"] == 0
+    assert np.abs(host(u) - exact).max() <= 1e-5 * max(np.abs(exact).max(), 1e-30)
