@@ -166,7 +166,9 @@ int draco_decode(draco_plan* plan, const void* R, const uint8_t* flags, float* u
  */
 int draco_decode_update(draco_plan* plan, const void* R, const uint8_t* flags, float* w, float scale, void* stream);
 
-/* locate + decode in one call (repetition: one pass over R; cyclic: locate, then decode). */
+/* locate + decode in one call.  Repetition: one pass over R.  Cyclic: three launches for short vectors (projection;
+ * one kernel for the sum of the block partials, the locator and the decode vector; recovery), one more (the
+ * reduction of the block partials) when the projection ran on more than 64 blocks.  f as in draco_locate. */
 int draco_locate_decode(draco_plan* plan, const void* R, const float* f, uint8_t* flags, float* u, void* stream);
 
 /* Repetition code with the selections exposed: maj (device [groups][d] fp32, may be NULL) receives
