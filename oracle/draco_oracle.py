@@ -287,52 +287,96 @@ def cyc_locate_from_projection(e: np.ndarray, q: np.ndarray, n: int, s: int, the
     nonfinite = ~(np.isfinite(e.real) & np.isfinite(e.imag) & np.isfinite(q))
     e[nonfinite] = 0.0
     q[nonfinite] = 0.0
-    out = _cyc_locate_finite(e, q, n, s, theta)
-    out["flags"] = out["flags"] | nonfinite
+    out = _cyc_locate_passes(e, q, n, s, theta, nonfinite)
     out["nonfinite"] = nonfinite
     return out
 
 
-def _cyc_locate_finite(e: np.ndarray, q: np.ndarray, n: int, s: int, theta: float) -> dict:
-    """The steps of phi on a finite projection record (see cyc_locate_from_projection)."""
+def _cyc_locate_passes(e: np.ndarray, q: np.ndarray, n: int, s: int, theta: float, known: np.ndarray) -> dict:
+    """phi on a finite projection record, run in passes.
+
+    The first pass is the paper's locator (syndromes, s x s Toeplitz system, recurrence, IDFT, support).
+    Reading where the paper is silent (it works in exact arithmetic, where one pass finds every adversary):
+    with complex64 vectors adversaries that sit close together on the circle make the system so badly
+    conditioned that a pass can miss some of them.  Every further pass therefore treats the set E of nodes
+    flagged so far as erasures: with lambda(x) = prod_{v in E} (x - w^v) = sum_k lambda_k x^k, the sequence
+    T_m = sum_k lambda_k h_{m-k} no longer contains the nodes of E (their terms carry the factor
+    lambda(w^v) = 0) and is again a sum of exponentials, one per adversary not yet flagged; the 2 s - |E|
+    values of T that the 2 s syndromes give (the last 2 s2 of them are used, s2 = floor((2 s - |E|) / 2))
+    go through the same system, recurrence and IDFT with s2 in place of s, and the nodes found join E.  The
+    passes end when one finds nothing (the usual second pass: its singular values are rounding noise) or
+    when fewer than two values of T are left.  Nodes known to be adversarial beforehand (``known``: a
+    non-finite record) are in E from the start, costing one syndrome each instead of two.  V can come out
+    as a superset of the adversaries (an honest node flagged by an ill-conditioned pass stays flagged);
+    decoding only needs V to contain them and |V| <= 2 s.  The rank cutoff of a pass is
+    theta * scale * sum_k |lambda_k| (the rounding noise of h enters T through those coefficients).
+
+    Returned ``t``, ``h``, ``sv``, ``beta``, ``margin`` are those of the first pass; ``rank`` is the number
+    of nodes the passes found (``ranks``: per pass).
+    """
     C = idft_matrix(n)
     scale = float(np.median(np.sqrt(np.asarray(q, dtype=np.float64))))
     tol = theta * scale
+    flags = np.asarray(known, dtype=bool).copy()
     out = {"e": e, "scale": scale, "t": np.zeros(n, dtype=np.complex128),
-           "flags": np.zeros(n, dtype=bool), "rank": 0, "h": np.zeros(n, dtype=np.complex128),
-           "margin": np.inf}
+           "flags": flags, "rank": 0, "h": np.zeros(n, dtype=np.complex128),
+           "margin": np.inf, "ranks": []}
     if s == 0:
         return out
+    w = np.exp(2j * np.pi / n)
     C_R = C[n - 2 * s:]
-    h = np.zeros(n, dtype=np.complex128)
-    h[n - 2 * s:] = e @ C_R.conj().T
-    out["h"] = h
-    M = np.empty((s, s), dtype=np.complex128)
-    rhs = np.empty(s, dtype=np.complex128)
-    for i in range(s):
-        for u in range(s):
-            M[i, u] = h[n - s - 1 - i + u]
-        rhs[i] = h[n - 1 - i]
-    Us, sv, Vh = np.linalg.svd(M)
-    keep = sv > tol
-    rank = int(np.count_nonzero(keep))
-    out["sv"] = sv
-    if rank == 0:
-        return out
-    inv = np.zeros_like(sv)
-    inv[keep] = 1.0 / sv[keep]
-    beta = Vh.conj().T @ (inv * (Us.conj().T @ rhs))
-    for ell in range(n - 2 * s):
-        acc = 0.0 + 0.0j
-        for u in range(s):
-            acc += beta[u] * h[(ell + u - s) % n]
-        h[ell] = acc
-    t = C @ h
-    order = np.argsort(-np.abs(t), kind="stable")
-    flags = np.zeros(n, dtype=bool)
-    flags[order[:rank]] = True
-    margin = np.abs(t[order[rank - 1]]) / max(np.abs(t[order[rank]]), 1e-300) if rank < n else np.inf
-    out.update(h=h, t=t, flags=flags, rank=rank, beta=beta, margin=float(margin))
+    syn = np.zeros(n, dtype=np.complex128)
+    syn[n - 2 * s:] = e @ C_R.conj().T                         # h_m, m = n-2s .. n-1
+    out["h"] = syn.copy()
+    first = True
+    while True:
+        E = np.flatnonzero(flags)
+        s2 = (2 * s - len(E)) // 2
+        if s2 < 1:
+            break
+        lam = np.ones(1, dtype=np.complex128)                  # lambda_k multiplies x^k
+        for v in E:                                            # times (x - w^v)
+            lam = np.concatenate([[0.0], lam]) - w ** v * np.concatenate([lam, [0.0]])
+        h = np.zeros(n, dtype=np.complex128)
+        for m in range(n - 2 * s2, n):
+            acc = 0.0 + 0.0j
+            for k in range(len(lam)):
+                acc += lam[k] * syn[m - k]
+            h[m] = acc
+        cut = tol * float(np.abs(lam).sum())
+        M = np.empty((s2, s2), dtype=np.complex128)
+        rhs = np.empty(s2, dtype=np.complex128)
+        for i in range(s2):
+            for u in range(s2):
+                M[i, u] = h[n - s2 - 1 - i + u]
+            rhs[i] = h[n - 1 - i]
+        Us, sv, Vh = np.linalg.svd(M)
+        keep = sv > cut
+        rank = int(np.count_nonzero(keep))
+        out["ranks"].append(rank)
+        if first:
+            out["sv"] = sv
+        if rank == 0:
+            break
+        inv = np.zeros_like(sv)
+        inv[keep] = 1.0 / sv[keep]
+        beta = Vh.conj().T @ (inv * (Us.conj().T @ rhs))
+        for ell in range(n - 2 * s2):
+            acc = 0.0 + 0.0j
+            for u in range(s2):
+                acc += beta[u] * h[(ell + u - s2) % n]
+            h[ell] = acc
+        t = C @ h
+        mag = np.abs(t)
+        mag[E] = -1.0                                          # already flagged: not candidates
+        order = np.argsort(-mag, kind="stable")
+        if first:
+            free = n - len(E)
+            margin = mag[order[rank - 1]] / max(mag[order[rank]], 1e-300) if rank < free else np.inf
+            out.update(h=h, t=t, beta=beta, margin=float(margin))
+        flags[order[:rank]] = True
+        out["rank"] += rank
+        first = False
     return out
 
 

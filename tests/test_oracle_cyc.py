@@ -144,22 +144,30 @@ def test_every_placement_of_up_to_s_adversaries_is_corrected(n, s):
 
 
 def test_failure_beyond_s():
-    """Theorem 1 / its corollary: s + 1 adversaries defeat a redundancy-(2 s + 1) code."""
+    """Theorem 1 / its corollary: s + 1 colluding adversaries defeat a redundancy-(2 s + 1) code.  The attack of the
+    proof: change one gradient g_k by delta; only the 2 s + 1 nodes that hold g_k send something else.  s + 1 of them
+    (the adversaries) send what they would send for the changed gradient, the other s stay honest.  The received
+    matrix is then s errors away from the coded vectors of the *changed* gradients, which is what any decoder must
+    return: the honest s get the blame and the sum is off by delta, with nothing to warn about."""
     n, s, d = 15, 2, 32
     G = di.gradient_rows(41, n, d)
     Z = orc.cyc_encode(G, n, s, dtype=np.complex128)
+    W = orc.cyc_W(n, s)
     f = di.projection_vector(42, d)
     exact = _exact_sum(G)
-    failures = 0
-    placements = list(itertools.combinations(range(n), s + 1))[::7]
-    for placement in placements:
-        R = Z.copy()
-        R[list(placement)] *= -100.0
-        out = orc.cyc_decode_full(R, f, n, s)
-        ok = (set(np.flatnonzero(out["flags"])) == set(placement) and out["u"] is not None
-              and np.abs(out["u"] - exact).max() <= 1e-6 * np.abs(exact).max())
-        failures += not ok
-    assert failures == len(placements)
+    delta = np.linspace(1.0, 2.0, d)
+    for k in (0, 6, 13):
+        holders = [(k + t) % n for t in range(2 * s + 1)]          # nodes j with W[k][j] != 0 (z_j uses g_{j-2s..j})
+        assert all(abs(W[k, j]) > 0 for j in holders) and np.count_nonzero(np.abs(W[k]) > 1e-12) == 2 * s + 1
+        for adversaries in itertools.combinations(holders, s + 1):
+            R = Z.copy()
+            for j in adversaries:
+                R[j] = Z[j] + W[k, j] * delta
+            out = orc.cyc_decode_full(R, f, n, s)
+            blamed = set(np.flatnonzero(out["flags"]))
+            assert blamed == set(holders) - set(adversaries)       # the honest holders of g_k
+            assert np.abs(out["u"] - (exact + delta)).max() <= 1e-9 * np.abs(exact).max()
+            assert np.abs(out["u"] - exact).max() >= 0.99
 
 
 def test_n4_any_two_coded_vectors_recover_the_sum():
@@ -341,3 +349,52 @@ def test_projection_and_energy_closed_forms():
     np.testing.assert_allclose(e2, want2, rtol=1e-11, atol=1e-11)
     # a transposed or conjugated operand would not pass: the ramp sum of row 1 has a non-zero imaginary part of known sign
     assert want2[1].imag < -1.0 and abs(e2[1].imag - want2[1].imag) < 1e-9
+
+
+def test_adjacent_adversaries_at_45_5_are_decoded_at_every_position():
+    """Definition 2 at the paper's own size with the worst placement for complex64 vectors: five adversaries side by
+    side, at each of the 45 positions on the circle.  One pass of the locator misses one of them in about half of the
+    positions (the 5 x 5 system's smallest singular value is a few times the cutoff); the passes with erasures find
+    a set that contains all five, at most 2 s nodes in all, and the sum comes out to the accuracy of the transport."""
+    n, s, d = 45, 5, 1024
+    W = orc.cyc_W(n, s)
+    worst = 0.0
+    supersets = 0
+    for start in range(n):
+        adv = [(start + k) % n for k in range(s)]
+        G = di.gradient_rows(1000 + start, n, d)
+        R = orc.cyc_encode(G, n, s, W=W)
+        di.apply_adversaries(R, adv, [di.ADV_REVGRAD] * s, [100.0] * s, seed=3)
+        f = di.projection_vector(2000 + start, d)
+        out = orc.cyc_decode_full(R, f, n, s)
+        found = set(np.flatnonzero(out["flags"]))
+        assert found >= set(adv) and len(found) <= 2 * s, (start, sorted(found))
+        supersets += found != set(adv)
+        exact = _exact_sum(G)
+        worst = max(worst, np.abs(out["u"] - exact).max() / np.abs(exact).max())
+    assert worst <= 2e-2, worst          # complex64 floor at (45, 5) is about 1.5e-3; a sixth erasure costs a little
+    assert supersets <= 15               # an honest node is blamed along with the five in about a quarter of the positions
+
+
+def test_known_bad_nodes_cost_one_syndrome_each():
+    """Nodes with a non-finite record are erasures from the start: s of them plus floor(s / 2) ordinary adversaries,
+    more than s nodes in all, are still all found and the sum is exact (2 s syndromes = erasures + 2 x errors)."""
+    import warnings
+    n, s, d = 15, 4, 64
+    G = di.gradient_rows(5, n, d)
+    Z = orc.cyc_encode(G, n, s)
+    f = di.projection_vector(6, d)
+    exact = _exact_sum(G)
+    rng = np.random.default_rng(0)
+    with warnings.catch_warnings():
+        warnings.simplefilter("ignore")
+        for trial in range(40):
+            nodes = rng.choice(n, s + s // 2, replace=False)
+            R = Z.copy()
+            for j in nodes[:s]:
+                R[j, int(rng.integers(0, d))] = np.nan
+            for j in nodes[s:]:
+                R[j] = -100 * R[j]
+            out = orc.cyc_decode_full(R, f, n, s)
+            assert set(np.flatnonzero(out["flags"])) == set(nodes.tolist())
+            assert np.abs(out["u"] - exact).max() <= 1e-4 * np.abs(exact).max()
