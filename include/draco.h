@@ -74,7 +74,7 @@ enum {
 typedef struct draco_info {
     int32_t status;        /* DRACO_OK, DRACO_ETOOMANY, DRACO_ENOMAJ or DRACO_EUNSURE */
     int32_t n_flagged;     /* |V|: nodes flagged by the last locate (or given to the last cyclic decode) */
-    int32_t locator_rank;  /* cyclic: numerical rank of the s x s syndrome system = adversaries seen */
+    int32_t locator_rank;  /* cyclic: adversaries seen = sum over the locator's passes of the numerical rank of the pass's system */
     int32_t n_active;      /* cyclic decode: number of rows with b_j != 0 */
     uint64_t no_majority;  /* repetition: (group, coordinate) pairs without a strict majority */
     double scale;          /* cyclic: median_j q_j^(1/2), q_j = sum_i |R[j][i]|^2: the unit of the rank cutoff */
@@ -138,8 +138,13 @@ int draco_encode(const draco_plan* plan, const float* G, void* Z, void* stream);
  *   cyclic:     V = phi(R): e = f R (fp64 accumulation), the 2 s syndromes e C_R^dagger,
  *               the s x s Toeplitz system for beta (pseudo-inverse solution from an SVD),
  *               the recurrence h_l = sum_u beta_u h_{l+u-s}, t = IDFT(h), V = supp(t)
- *               read as the rank-many largest |t_j|.  A node whose vector holds NaN or infinities (its
- *               projection is then not finite) is flagged outright and counted as having sent f R_j = 0.
+ *               read as the rank-many largest |t_j|.  That is one pass; further passes treat the nodes
+ *               flagged so far as erasures (modified syndromes sum_k lambda_k h_{m-k}, lambda(x) =
+ *               prod_{v in V} (x - w^v)) and look for more in the same way, until a pass finds nothing:
+ *               adversaries side by side, which one pass cannot always separate with complex64 vectors, end
+ *               up in V all the same, at times together with an honest neighbour (V then is a superset of
+ *               the adversaries, which is all that decoding needs, as long as |V| <= 2 s).  A node whose
+ *               vector holds NaN or infinities (its projection is then not finite) is in V from the start.
  * R: device [n][d].  f: device [d] fp32, the caller's draw of N(1_d, I_d) (cyclic only).
  * flags: device [n] bytes.
  */

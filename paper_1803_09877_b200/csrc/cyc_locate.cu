@@ -825,46 +825,116 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, const double2*
     }
     __syncthreads();
     const double tol = theta * scale_s;
-    int rank = 0;
-    bool flagged = false;
+    // The locator runs in passes.  The first is the paper's phi.  Each further pass treats the set E of nodes flagged
+    // so far (nodes with a non-finite record from the start) as erasures: with lambda(x) = prod_{v in E} (x - w^v) =
+    // sum_k lambda_k x^k the sequence T_m = sum_k lambda_k h_{m-k} no longer contains the nodes of E and is again a sum
+    // of exponentials, one per adversary not yet flagged, so its last 2 s2 values, s2 = floor((2 s - |E|) / 2), go
+    // through the same Toeplitz system, recurrence and IDFT with s2 in place of s.  A pass that finds nothing (the
+    // usual second pass: rounding noise) ends the search.  Adversaries that sit side by side make one pass miss some of
+    // them with complex64 vectors; the passes then still end with a set that contains them all.
+    __shared__ double2 syn[kMaxN];                         // h_{n-2s+i}: every pass rewrites h
+    __shared__ double2 lam[kMaxN + 2];
+    __shared__ uint8_t fl_s[kMaxN];                        // V so far
+    __shared__ int elist[kMaxN];
+    __shared__ int eps_s, rank_total_s, sweeps_s;
+    __shared__ double lam1_s, margin_s;
+    if (tid < 2 * s) syn[tid] = h[n - 2 * s + tid];
+    if (tid < n) {
+        fl_s[tid] = nonfinite[tid];
+        cd->t[tid] = make_double2(0.0, 0.0);
+        cd->h[tid] = h[tid];
+    }
+    if (tid == 0) { rank_total_s = 0; sweeps_s = 0; margin_s = 1e300; }
+    __syncthreads();
     double2* beta = beta_s;
-    if (s > 0) {
-        // row i: [h_{n-s-1-i} .. h_{n-2-i}] beta = h_{n-1-i}; stored by columns
-        const int sp = s + (s & 1);
-        const bool small = sp <= kSmallDim;
-        double2* A = small ? As : cd->work;
-        double2* V = small ? Vs : cd->work + sp * sp;
-        for (int idx = tid; idx < sp * sp; idx += blockDim.x) {
-            const int c = idx / sp, i = idx % sp;
-            A[idx] = (c < s && i < s) ? h[n - s - 1 - i + c] : make_double2(0.0, 0.0);
+    bool first = true;
+    for (int pass = 0; pass <= 2 * s && s > 0; ++pass) {
+        if (tid == 0) {
+            int a = 0;
+            for (int j = 0; j < n; ++j)
+                if (fl_s[j]) elist[a++] = j;
+            eps_s = a;
         }
-        if (tid < s) rhs_s[tid] = h[n - 1 - tid];
         __syncthreads();
-        // No singular value exceeds the Frobenius norm: when that is within the cutoff (the usual step without any
-        // adversary, where the syndromes are rounding noise) the rank is 0 and the SVD is skipped.
+        const int eps = eps_s;
+        const int s2 = (2 * s - eps) / 2;
+        if (s2 < 1) break;
+        // lambda: one factor (x - w^v) at a time, new_k = old_{k-1} - w^v old_k
+        if (tid <= eps) lam[tid] = make_double2(tid == 0 ? 1.0 : 0.0, 0.0);
+        __syncthreads();
+        for (int a = 0; a < eps; ++a) {
+            double2 nv = make_double2(0.0, 0.0);
+            if (tid <= a + 1) {
+                const double2 wv = tw[elist[a]];
+                const double2 prev = tid > 0 ? lam[tid - 1] : make_double2(0.0, 0.0);
+                const double2 cur = tid <= a ? lam[tid] : make_double2(0.0, 0.0);
+                const double2 q = cmul(wv, cur);
+                nv = make_double2(prev.x - q.x, prev.y - q.y);
+            }
+            __syncthreads();
+            if (tid <= a + 1) lam[tid] = nv;
+            __syncthreads();
+        }
         if (tid < 32) {
-            double fro2 = 0.0;
-            for (int idx = tid; idx < sp * sp; idx += 32) fro2 += cabs2(A[idx]);
-            fro2 = warp_sum(fro2);
-            if (tid == 0) sh[2] = (fro2 > tol * tol) ? 1 : 0;
+            double acc = 0.0;
+            for (int k = tid; k <= eps; k += 32) acc += sqrt(cabs2(lam[k]));
+            acc = warp_sum(acc);
+            if (tid == 0) lam1_s = acc;
+        }
+        if (tid < n) {                                     // T_m on its window m = n - 2 s2 .. n - 1, zero before it
+            double a = 0.0, b = 0.0;
+            if (tid >= n - 2 * s2)
+                for (int k = 0; k <= eps; ++k) {
+                    const double2 q = cmul(lam[k], syn[tid - k - (n - 2 * s)]);
+                    a += q.x;
+                    b += q.y;
+                }
+            h[tid] = make_double2(a, b);
         }
         __syncthreads();
-        if (sh[2]) {
-            if (small) {
-                if (tid < 32) warp_jacobi_pinv(A, V, rhs_s, s, tol, beta_s, coef_s, sh);
-                __syncthreads();
-                rank = sh[1];
-            } else {
-                rank = block_jacobi_pinv(A, V, rhs_s, s, tol, beta_s, coef_s, sh);
+        const double cut = tol * lam1_s;                   // the rounding noise of h enters T through |lambda_k|
+        int rank = 0;
+        {
+            // row i: [h_{n-s2-1-i} .. h_{n-2-i}] beta = h_{n-1-i}; stored by columns
+            const int sp = s2 + (s2 & 1);
+            const bool small = sp <= kSmallDim;
+            double2* A = small ? As : cd->work;
+            double2* V = small ? Vs : cd->work + sp * sp;
+            for (int idx = tid; idx < sp * sp; idx += blockDim.x) {
+                const int c = idx / sp, i = idx % sp;
+                A[idx] = (c < s2 && i < s2) ? h[n - s2 - 1 - i + c] : make_double2(0.0, 0.0);
+            }
+            if (tid < s2) rhs_s[tid] = h[n - 1 - tid];
+            __syncthreads();
+            // No singular value exceeds the Frobenius norm: when that is within the cutoff (the usual step without any
+            // adversary, and the usual last pass: rounding noise) the rank is 0 and the SVD is skipped.
+            if (tid < 32) {
+                double fro2 = 0.0;
+                for (int idx = tid; idx < sp * sp; idx += 32) fro2 += cabs2(A[idx]);
+                fro2 = warp_sum(fro2);
+                if (tid == 0) sh[2] = (fro2 > cut * cut) ? 1 : 0;
+            }
+            __syncthreads();
+            if (sh[2]) {
+                if (small) {
+                    if (tid < 32) warp_jacobi_pinv(A, V, rhs_s, s2, cut, beta_s, coef_s, sh);
+                    __syncthreads();
+                    rank = sh[1];
+                } else {
+                    rank = block_jacobi_pinv(A, V, rhs_s, s2, cut, beta_s, coef_s, sh);
+                }
+                if (tid == 0) {                            // sweeps of the longest iteration; negative once one hit the limit
+                    if (sh[3] < 0) sweeps_s = sh[3];
+                    else if (sweeps_s >= 0 && sh[3] > sweeps_s) sweeps_s = sh[3];
+                }
             }
         }
-    }
-    if (rank > 0) {
+        if (rank == 0) break;
         if (tid == 0) {
-            for (int l = 0; l < n - 2 * s; ++l) {
+            for (int l = 0; l < n - 2 * s2; ++l) {
                 double a = 0.0, b = 0.0;
-                for (int u = 0; u < s; ++u) {
-                    int idx = l + u - s;
+                for (int u = 0; u < s2; ++u) {
+                    int idx = l + u - s2;
                     if (idx < 0) idx += n;
                     const double2 q = cmul(beta[u], h[idx]);
                     a += q.x;
@@ -885,24 +955,35 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, const double2*
                 if (idx >= n) idx -= n;
             }
             const double2 t = make_double2(a * rsn, b * rsn);
-            cd->t[tid] = t;
-            mag[tid] = cabs2(t);
+            if (first) {
+                cd->t[tid] = t;
+                cd->h[tid] = h[tid];
+            }
+            mag[tid] = fl_s[tid] ? -1.0 : cabs2(t);        // nodes already in V are not candidates
         }
         __syncthreads();
-        // exactly `rank` entries of t are non-zero in exact arithmetic: V = the rank largest |t_j|
+        // exactly `rank` entries of t are non-zero in exact arithmetic: the rank largest |t_j| join V
+        bool found = false;
         if (tid < n) {
             int pos = 0;
             for (int k = 0; k < n; ++k) pos += (mag[k] > mag[tid]) || (mag[k] == mag[tid] && k < tid);
-            flagged = pos < rank;
-            if (pos == rank - 1) sorted[0] = mag[tid];     // |t|^2 of the weakest flagged node ..
-            if (pos == rank) sorted[1] = mag[tid];         // .. and of the strongest unflagged one
+            found = pos < rank;
+            if (first && pos == rank - 1) sorted[0] = mag[tid];     // |t|^2 of the weakest flagged node ..
+            if (first && pos == rank) sorted[1] = mag[tid];         // .. and of the strongest unflagged one
         }
-    } else if (tid < n) {
-        cd->t[tid] = make_double2(0.0, 0.0);
+        __syncthreads();
+        if (found) fl_s[tid] = 1;
+        if (tid == 0) {
+            rank_total_s += rank;
+            if (first && rank < n - eps) margin_s = sqrt(sorted[0] / fmax(sorted[1], 1e-300));
+        }
+        first = false;
+        __syncthreads();
     }
+    __syncthreads();
+    bool flagged = false;
     if (tid < n) {
-        cd->h[tid] = h[tid];
-        flagged = flagged || nonfinite[tid];
+        flagged = fl_s[tid] != 0;
         if (flags) flags[tid] = flagged ? 1 : 0;
         if (flags2) flags2[tid] = flagged ? 1 : 0;
         if (flagged) atomicAdd(&count, 1);
@@ -910,21 +991,19 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, const double2*
     __syncthreads();
     if (tid == 0) {
         info->n_flagged = count;
-        info->locator_rank = rank;
+        info->locator_rank = rank_total_s;
         info->scale = scale_s;
         info->max_syndrome = maxsyn_s;
-        const double margin = (rank > 0 && rank < n) ? sqrt(sorted[0] / fmax(sorted[1], 1e-300)) : 1e300;
+        const double margin = margin_s;
         // exactly `rank` entries of t are non-zero in exact arithmetic: where the weakest flagged and the strongest
-        // unflagged |t_j| are less than a decade apart the choice of V is not to be trusted, nor is a rank that comes
-        // from an iteration that was stopped at its sweep limit (NaN in R makes the comparison false: unsure)
-        info->status = (margin >= kMarginBar && sh[3] >= 0) ? DRACO_OK : DRACO_EUNSURE;
+        // unflagged |t_j| of the first pass are less than a decade apart the choice of V is not to be trusted, nor is a
+        // rank that comes from an iteration that was stopped at its sweep limit
+        info->status = (margin >= kMarginBar && sweeps_s >= 0) ? DRACO_OK : DRACO_EUNSURE;
         info->no_majority = 0;
         info->locator_margin = margin;
-        info->svd_sweeps = sh[3];
+        info->svd_sweeps = sweeps_s;
     }
     if (with_b) {                                          // the decode vector for the V just found, same launch
-        __shared__ uint8_t fl_s[kMaxN];
-        if (tid < n) fl_s[tid] = flagged ? 1 : 0;
         __syncthreads();
         decode_vector_body(cd, fl_s, n, s, info);
     }
