@@ -17,12 +17,14 @@ is exceeded (Theorem 1); the hand-derived n=4, s=1 coefficient table; Lemma 3
 (support of W, 1_P in the span); Lemma 7 (C_L C_R^dagger = 0, clean syndromes
 vanish); the locator returning t = (f N)^T value for value (proof of Lemma 4);
 Algorithm 2 against sort-and-count; the adversary-free decode reducing to a
-plain sum.
+plain sum; NaN / infinite vectors and five adjacent adversaries at n = 45
+decoded at every placement; the colluding attack of Theorem 1's proof.
 
 Parity unpinned (readings, not paper facts; they do not change the exact
 result): the rank cutoff ``theta`` of the locator and its "rank largest |t_j|"
 reading of t_j != 0; the grouping used when 2 s + 1 does not divide n; the
-minimum-norm choice among the valid decode vectors b.
+minimum-norm choice among the valid decode vectors b; the cutoff of the locator's
+later passes (theta * scale * sum |lambda_k|).
 """
 from __future__ import annotations
 
