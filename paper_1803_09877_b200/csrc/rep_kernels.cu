@@ -355,7 +355,7 @@ int launch_rep_encode(const draco_plan* p, const float* G, float* Z, int64_t len
         if (gt.max_size <= 3) DRACO_ENC(3, 4, 5);
         else if (gt.max_size <= 4) DRACO_ENC(4, 4, 4);
         else if (gt.max_size <= 5) DRACO_ENC(5, 4, 2);
-        else if (gt.max_size <= 8) DRACO_ENC(8, 4, 2);
+        else if (gt.max_size <= 8) DRACO_ENC(8, 4, 1);
         else if (gt.max_size <= 16) DRACO_ENC(16, 4, 1);
         else DRACO_ENC(0, 4, 1);
     } else {
