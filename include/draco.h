@@ -65,8 +65,9 @@ enum {
                             an imaginary part above 1e-2 of its real part (im_residual, re_max), or the singular-value
                             iteration of the syndrome system stopped at its sweep limit (svd_sweeps < 0).  More than s
                             adversaries, or adversaries that the precision of complex64 vectors cannot separate, show up
-                            here; u is still written.  (A low locator_margin next to a small im_residual after the decode
-                            means that the locator's later passes repaired what its first pass left open: the sum is good) */
+                            here; u is still written.  Once an unpacked plan has decoded, im_residual decides: a low
+                            locator_margin next to a clean residual means that the locator's later passes closed what its
+                            first pass left open, and the status is DRACO_OK; packed plans have no residual to go by */
 };
 
 #define DRACO_MAX_N 128  /* largest supported number of nodes */

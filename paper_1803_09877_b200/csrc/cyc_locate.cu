@@ -1002,6 +1002,8 @@ cyc_solve_kernel(CycDevice* cd, const double2* __restrict__ e_in, const double2*
         info->no_majority = 0;
         info->locator_margin = margin;
         info->svd_sweeps = sweeps_s;
+        info->im_residual_bits = 0ull;                     // a decode's self-check belongs to the locate before it
+        info->re_max_bits = 0ull;
     }
     if (with_b) {                                          // the decode vector for the V just found, same launch
         __syncthreads();

@@ -320,8 +320,17 @@ int draco_get_info(draco_plan* plan, draco_info* info, void* stream) {
     // The recovery kernel's blocks only merge their maxima; the verdict on them is formed here.  u-hat = G 1_P is
     // real: an imaginary part beyond rounding means an adversary is still among the rows that were combined.
     // (NaN from an adversary compares false with everything and so counts as a failed check.)
-    if (is_cyc(plan) && info->status == DRACO_OK && !(info->im_residual <= kImResidualBar * info->re_max))
-        info->status = DRACO_EUNSURE;
+    if (is_cyc(plan) && (info->status == DRACO_OK || info->status == DRACO_EUNSURE)) {
+        const bool decoded = info->re_max > 0.0 || info->im_residual > 0.0 || info->re_max != info->re_max;   // since the last locate
+        const bool residual_ok = info->im_residual <= kImResidualBar * info->re_max;
+        if (decoded && !residual_ok) {
+            info->status = DRACO_EUNSURE;
+        } else if (decoded && info->status == DRACO_EUNSURE && info->svd_sweeps >= 0 && !is_packed(plan)) {
+            // the only open point was the first pass's margin, and the decode's own check came out clean: the
+            // locator's later passes closed it (adversaries side by side; V then holds them all)
+            info->status = DRACO_OK;
+        }
+    }
     return h.internal_error ? DRACO_EINTERNAL : DRACO_OK;
 }
 

@@ -658,4 +658,5 @@ def test_adjacent_adversaries_at_45_5():
         exact = G.astype(np.float64).sum(axis=0)
         assert normwise(host(u), exact) <= 2e-2, start
         assert info["im_residual"] <= 1e-2 * info["re_max"]          # nobody adversarial is left among the rows combined
+        assert info["status"] == 0                                   # whatever the first pass's margin was
     assert supersets >= 1                                            # at least one of these positions needs the extra pass

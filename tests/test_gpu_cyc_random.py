@@ -44,10 +44,16 @@ def test_random_small_cases_match_the_oracle(stream_seed):
         want = orc.cyc_locate(R, f, n, s)
         what = f"case {case}: n={n} s={s} adv={adv} model={model} d={d} seed={seed}"
         tol = 1e-6 * want["scale"]
-        # whatever the locator made of it: a set that is not the planted one never comes back as DRACO_OK
-        if sorted(np.flatnonzero(host(flags)).tolist()) != adv:
+        # whatever the locator made of it: a set that misses an adversary never comes back as DRACO_OK, and a set that
+        # holds them all (plus an honest node flagged along by a hard pass) gives the right sum
+        got = set(np.flatnonzero(host(flags)).tolist())
+        if got != set(adv):
             warned += 1
-            assert info["status"] in (dr.binding.EUNSURE, dr.binding.ETOOMANY), what
+            if got >= set(adv) and len(got) <= 2 * s:
+                exact = G.astype(np.float64).sum(axis=0)
+                assert normwise(host(u), exact) <= 5e-2, what
+            else:
+                assert info["status"] in (dr.binding.EUNSURE, dr.binding.ETOOMANY), what
         if any(tol / 3 < x < 3 * tol for x in want.get("sv", [])) or (0 < want["rank"] < n and want["margin"] < 10):
             on_the_edge += 1         # a singular value at the rank cutoff, or |t| of flagged and unflagged nodes alike: counted
         np.testing.assert_array_equal(host(flags).astype(bool), want["flags"], err_msg=what)
